@@ -1,0 +1,247 @@
+"""Seeded synthetic workloads: tensor shapes and value generators for the five configurations.
+
+This module holds NO arithmetic of the optimizer step. It only decides shapes, lays tensors out in
+flat buffers and fills parameters and gradients with seeded random values, so it can serve both the
+CUDA path and the CPU checker without making them share code of the method.
+
+The workloads stand in for the paper's Qwen-family fine-tuning runs (Sec. 4 setup and the training
+configuration table): only parameter shapes and value distributions are used, no dataset or weights.
+
+Recipes
+  tiny    8 fp32 tensors [512,512]x4, [512,2048]x2, [2048,512], [512]; p ~ N(0, 0.02^2);
+          g ~ N(0, (1e-3)^2) rounded to bf16, step-2 gradients scaled by 1e3; seed 0.
+  ragged  1000 fp32 tensors packed back to back (bases are element-aligned only);
+          size = floor(exp(U(0, ln max_numel))), with probability 0.70 rounded to the nearest positive
+          multiple of 2048, else forced off a multiple of 2048; 5 % of tensors have all-zero
+          gradients every step; g ~ 1e-3 * Student-t(3) rounded to bf16; seed 1.
+  3b      Qwen2.5-3B-shaped list (hidden 2048, 36 layers, 16 q / 2 kv heads of 128, intermediate
+          11008, vocab 151936 tied): fp32 params, bf16 grads ~ N(0, s_l^2) with
+          s_l = 1e-4 * 10^(u_l - 0.5), u_l ~ U(0,1) per layer; seed 2.
+  7b      Qwen2.5-7B-shaped list (hidden 3584, 28 layers, 28 / 4 heads, intermediate 18944, vocab
+          152064 untied): fp32 params, bf16 grads ~ N(0, (1e-4)^2); seed 3.
+  27b     dense decoder (hidden 5120, 56 layers, 40 / 8 heads, intermediate 25600, vocab 151936
+          untied): bf16 params, bf16 grads ~ N(0, (5e-5)^2); seed 4.
+Norm weights are initialised to 1, every other parameter ~ N(0, 0.02^2).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+HEAD_DIM = 128
+
+
+@dataclass
+class Spec:
+    name: str
+    names: List[str]
+    sizes: List[int]
+    layer_of: List[int]              # layer index per tensor (-1: not in a decoder layer)
+    param_dtype: torch.dtype
+    grad_dtype: torch.dtype = torch.bfloat16
+    seed: int = 0
+    grad_std: float = 1e-3
+    grad_kind: str = "normal"        # "normal" | "student3" | "layer_normal"
+    zero_grad_frac: float = 0.0
+    max_norm: float = 1.0
+    steps: int = 3
+    step_scale: dict = field(default_factory=dict)   # {step: factor} applied to that step's grads
+    align_elems: int = 1             # each tensor's offset in the flat buffers is a multiple of this
+
+    @property
+    def numel(self) -> int:
+        return int(sum(self.sizes))
+
+    def n_blocks(self, block: int) -> int:
+        return int(sum((s + block - 1) // block for s in self.sizes))
+
+
+def _decoder(name, hidden, layers, q_heads, kv_heads, inter, vocab, tied, **kw) -> Spec:
+    names, sizes, layer_of = [], [], []
+
+    def add(n, s, l):
+        names.append(n); sizes.append(int(s)); layer_of.append(l)
+
+    add("embed", vocab * hidden, -1)
+    for l in range(layers):
+        add(f"l{l}.q_proj", q_heads * HEAD_DIM * hidden, l)
+        add(f"l{l}.k_proj", kv_heads * HEAD_DIM * hidden, l)
+        add(f"l{l}.v_proj", kv_heads * HEAD_DIM * hidden, l)
+        add(f"l{l}.o_proj", hidden * q_heads * HEAD_DIM, l)
+        add(f"l{l}.gate_proj", inter * hidden, l)
+        add(f"l{l}.up_proj", inter * hidden, l)
+        add(f"l{l}.down_proj", hidden * inter, l)
+        add(f"l{l}.input_norm", hidden, l)
+        add(f"l{l}.post_attn_norm", hidden, l)
+    add("final_norm", hidden, -1)
+    if not tied:
+        add("lm_head", vocab * hidden, -1)
+    return Spec(name=name, names=names, sizes=sizes, layer_of=layer_of, align_elems=16, **kw)
+
+
+def tiny_spec() -> Spec:
+    shapes = [(512, 512)] * 4 + [(512, 2048)] * 2 + [(2048, 512), (512,)]
+    sizes = [int(np.prod(s)) for s in shapes]
+    return Spec("tiny", [f"t{i}" for i in range(len(sizes))], sizes, [-1] * len(sizes), torch.float32,
+                seed=0, grad_std=1e-3, grad_kind="normal", max_norm=1.0, steps=3, step_scale={2: 1e3},
+                align_elems=16)
+
+
+def ragged_spec(n_tensors: int = 1000, max_numel: int = 4 << 20, seed: int = 1, multiple: int = 2048) -> Spec:
+    rng = np.random.default_rng(seed)
+    sizes = []
+    for _ in range(n_tensors):
+        s = int(math.floor(math.exp(rng.uniform(0.0, math.log(max_numel)))))
+        s = max(1, min(s, max_numel))
+        if rng.uniform() < 0.70:
+            s = max(multiple, int(round(s / multiple)) * multiple)
+        elif s % multiple == 0:
+            s += 1 + int(rng.integers(0, multiple - 1))
+        sizes.append(s)
+    return Spec("ragged", [f"r{i}" for i in range(n_tensors)], sizes, [-1] * n_tensors, torch.float32,
+                seed=seed, grad_std=1e-3, grad_kind="student3", zero_grad_frac=0.05, max_norm=0.5,
+                steps=10, align_elems=1)
+
+
+def qwen3b_spec() -> Spec:
+    return _decoder("3b", 2048, 36, 16, 2, 11008, 151936, True, param_dtype=torch.float32, seed=2,
+                    grad_std=1e-4, grad_kind="layer_normal", max_norm=1.0, steps=1)
+
+
+def qwen7b_spec() -> Spec:
+    return _decoder("7b", 3584, 28, 28, 4, 18944, 152064, False, param_dtype=torch.float32, seed=3,
+                    grad_std=1e-4, grad_kind="normal", max_norm=1.0, steps=5)
+
+
+def dense27b_spec() -> Spec:
+    return _decoder("27b", 5120, 56, 40, 8, 25600, 151936, False, param_dtype=torch.bfloat16, seed=4,
+                    grad_std=5e-5, grad_kind="normal", max_norm=1.0, steps=3)
+
+
+def scaled_decoder_spec(name: str, hidden: int, layers: int, q_heads: int, kv_heads: int, inter: int,
+                        vocab: int, tied: bool, param_dtype=torch.float32, seed: int = 7,
+                        grad_std: float = 1e-4, grad_kind: str = "layer_normal") -> Spec:
+    """A decoder-shaped list with caller-chosen dimensions (small cases for tests and profiling)."""
+    return _decoder(name, hidden, layers, q_heads, kv_heads, inter, vocab, tied, param_dtype=param_dtype,
+                    seed=seed, grad_std=grad_std, grad_kind=grad_kind, max_norm=1.0, steps=1)
+
+
+SPECS = {"tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
+
+
+def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:
+    """Tensor indices grouped for chunked update: non-layer tensors first, then runs of layers."""
+    groups = [[i for i, l in enumerate(spec.layer_of) if l < 0]]
+    n_layers = max(spec.layer_of) + 1 if spec.layer_of else 0
+    for l0 in range(0, n_layers, layers_per_group):
+        groups.append([i for i, l in enumerate(spec.layer_of) if l0 <= l < l0 + layers_per_group])
+    return [g for g in groups if g]
+
+
+class Buffers:
+    """Flat device (or host) buffers for one workload; tensor t occupies [off[t], off[t]+size[t]) of
+    param / grad / m_code / v_code and [boff[t], boff[t]+nb[t]) of the two scale arrays."""
+
+    def __init__(self, spec: Spec, block: int, device, pin: bool = False):
+        self.spec, self.block, self.device = spec, int(block), torch.device(device)
+        a = spec.align_elems
+        self.off, self.boff = [], []
+        o = b = 0
+        for s in spec.sizes:
+            o = (o + a - 1) // a * a
+            self.off.append(o); self.boff.append(b)
+            o += s; b += (s + block - 1) // block
+        self.total, self.total_blocks = o, b
+        kw = dict(device=self.device)
+        if pin and self.device.type == "cpu":
+            kw["pin_memory"] = True
+        self.param = torch.empty(max(o, 1), dtype=spec.param_dtype, **kw)
+        self.grad = torch.empty(max(o, 1), dtype=spec.grad_dtype, **kw)
+        self.m_code = torch.empty(max(o, 1), dtype=torch.uint8, **kw)
+        self.v_code = torch.empty(max(o, 1), dtype=torch.uint8, **kw)
+        self.m_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
+        self.v_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
+
+    def view(self, which: str, t: int) -> torch.Tensor:
+        buf = getattr(self, which)
+        if which in ("m_absmax", "v_absmax"):
+            nb = (self.spec.sizes[t] + self.block - 1) // self.block
+            return buf[self.boff[t]: self.boff[t] + nb]
+        return buf[self.off[t]: self.off[t] + self.spec.sizes[t]]
+
+    def resident_bytes(self) -> int:
+        return sum(getattr(self, k).numel() * getattr(self, k).element_size()
+                   for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax"))
+
+
+def _gen(device, seed: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def fill_params(buf: Buffers) -> None:
+    """p ~ N(0, 0.02^2); tensors whose name ends in 'norm' are set to 1."""
+    spec = buf.spec
+    gen = _gen(buf.device, spec.seed * 1000 + 1)
+    if buf.total > sum(spec.sizes):
+        buf.param.zero_()
+    for t, name in enumerate(spec.names):
+        v = buf.view("param", t)
+        if name.endswith("norm"):
+            v.fill_(1.0)
+        else:
+            v.normal_(0.0, 0.02, generator=gen)
+
+
+def layer_stds(spec: Spec) -> List[float]:
+    """Per-tensor gradient standard deviation (layer_normal: one draw per layer, 10x spread)."""
+    if spec.grad_kind != "layer_normal":
+        return [spec.grad_std] * len(spec.sizes)
+    rng = np.random.default_rng(spec.seed * 1000 + 7)
+    n_layers = max(spec.layer_of) + 1
+    u = rng.uniform(0.0, 1.0, n_layers + 1)
+    return [spec.grad_std * 10.0 ** (u[l if l >= 0 else n_layers] - 0.5) for l in spec.layer_of]
+
+
+def zero_grad_mask(spec: Spec) -> List[bool]:
+    rng = np.random.default_rng(spec.seed * 1000 + 3)
+    return [bool(rng.uniform() < spec.zero_grad_frac) for _ in spec.sizes]
+
+
+def fill_grads(buf: Buffers, step: int, max_chunk: int = 1 << 26) -> None:
+    """Fresh gradients for optimizer step `step` (1-based), reproducible per (seed, step)."""
+    spec = buf.spec
+    gen = _gen(buf.device, spec.seed * 1000 + 100 + step)
+    stds = layer_stds(spec)
+    zeros = zero_grad_mask(spec)
+    scale = float(spec.step_scale.get(step, 1.0))
+    if buf.total > sum(spec.sizes):
+        buf.grad.zero_()
+    for t in range(len(spec.sizes)):
+        v = buf.view("grad", t)
+        if zeros[t]:
+            v.zero_()
+            continue
+        if spec.grad_kind == "student3":
+            for a in range(0, v.numel(), max_chunk):
+                w = v[a: a + max_chunk]
+                z = torch.empty(4, w.numel(), dtype=torch.float32, device=buf.device)
+                z.normal_(0.0, 1.0, generator=gen)
+                tval = z[0] / torch.sqrt((z[1] * z[1] + z[2] * z[2] + z[3] * z[3]) / 3.0)
+                w.copy_((tval * (stds[t] * scale)).to(spec.grad_dtype))
+        else:
+            v.normal_(0.0, stds[t] * scale, generator=gen)
+
+
+def numpy_view(t: torch.Tensor) -> np.ndarray:
+    """Host numpy array sharing memory with a CPU tensor (bf16 as its uint16 bit pattern)."""
+    t = t.detach()
+    assert t.device.type == "cpu"
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()
