@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the fused clip + block-wise 8-bit AdamW optimizer step on B200.
+
+One "step" = one pass of the whole hot path over the workload: zero the norm scalar, multi-tensor
+squared gradient norm (all chunks), fused dequantize/clip/AdamW/requantize step (all chunks), all on
+one stream with no host synchronisation. Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workloads 7b,3b,27b] [--block 2048]
+    python bench.py --impl reference ...        # the CPU oracle, timed on a bounded sample
+
+At N > 1 (torchrun) every rank owns a full copy of the headline workload as its shard of an N-times
+larger model; the only exchange is a sum all-reduce of the 8-byte squared norm between the norm
+and the step (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "optimizer-step params/s"
+UNIT = "params/s"
+# DRAM bytes per parameter of the fused step kernel measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum over one launch / parameters of that launch); see profiles/. None = not captured.
+STEP_TRAFFIC_BYTES_PER_PARAM = {"f32": None, "bf16": None}
+
+
+def algorithmic_bytes_per_param(param_bytes: int, block: int):
+    """(norm kernel, step kernel) bytes per parameter the method itself must move."""
+    norm = 2.0                                   # read bf16 gradient once
+    step = 2.0 * param_bytes + 2.0 + 2.0 + 2.0 + 16.0 / block   # p r/w, g, codes r, codes w, scales r/w
+    return norm, step
+
+
+def measured_peak_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.1] or [l for (_, l) in self.lines[-3:]]
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(name: str, block: int, device):
+    import torch
+    import paper_2608_11919_b200 as L
+    from paper_2608_11919_b200 import workloads as W
+    spec = W.SPECS[name]()
+    buf = W.Buffers(spec, block, device)
+    W.fill_params(buf)
+    W.fill_grads(buf, 1)
+    tl = L.TensorList.from_buffers(buf)
+    chunks = None
+    if len(spec.sizes) > 480 or name == "27b":        # layer-group chunks under one global clip norm
+        chunks = [L.TensorList.from_buffers(buf, g) for g in W.layer_groups(spec, 8)]
+    opt = L.Hybrid8Optimizer(tl, block, L.HParams(max_norm=spec.max_norm), chunks)
+    opt.init_state()
+    torch.cuda.synchronize()
+    return spec, buf, opt
+
+
+def one_step(opt, L, dist_on, ev=None):
+    """Enqueue one optimizer step; ev = (e0, e1, e2) CUDA events to record around norm and step."""
+    import torch
+    opt.t += 1
+    opt.hp.step = opt.t
+    opt.sqnorm.zero_()
+    if ev:
+        ev[0].record()
+    for ch in opt.chunks:
+        L.lt_grad_sqnorm_multi(ch, opt.sqnorm, opt.workspace)
+    if ev:
+        ev[1].record()
+    if dist_on:
+        torch.distributed.all_reduce(opt.sqnorm)
+    if ev:
+        ev[2].record()
+    for ch in opt.chunks:
+        L.lt_hybrid8_step(ch, opt.block, opt.hp, opt.sqnorm, opt.status)
+    if ev:
+        ev[3].record()
+
+
+def time_resident(name, block, steps, warmup, rank, world, dist_on, sample_clocks):
+    import torch
+    import paper_2608_11919_b200 as L
+    dev = torch.device("cuda", torch.cuda.current_device())
+    spec, buf, opt = build_workload(name, block, dev)
+    N = spec.numel
+    for _ in range(max(warmup, 3)):
+        one_step(opt, L, dist_on)
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device()) if sample_clocks else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    start.record()
+    for k in range(steps):
+        one_step(opt, L, dist_on, evs[k])
+    end.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    if dist_on:
+        torch.distributed.barrier()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    total_ms = start.elapsed_time(end)
+    norm_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    step_ms = [e[2].elapsed_time(e[3]) for e in evs]
+    status = int(opt.status.item())
+    if dist_on:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    pbytes = 2 if spec.param_dtype == torch.bfloat16 else 4
+    nb, sb = algorithmic_bytes_per_param(pbytes, block)
+    n_chunks = len(opt.chunks)
+    res = {
+        "workload": name, "params": N, "tensors": len(spec.sizes), "chunks": n_chunks,
+        "param_dtype": "bf16" if pbytes == 2 else "f32", "resident_gb": round(buf.resident_bytes() / 1e9, 2),
+        "ms_per_step": total_ms / steps, "params_per_s": N * world / (total_ms / steps * 1e-3),
+        "norm_ms": statistics.mean(norm_ms), "step_ms": statistics.mean(step_ms),
+        "norm_gbs": N * nb / (statistics.mean(norm_ms) * 1e-3) / 1e9,
+        "step_gbs": N * sb / (statistics.mean(step_ms) * 1e-3) / 1e9,
+        "whole_gbs": N * (nb + sb) / (total_ms / steps * 1e-3) / 1e9,
+        "step_ms_min": min(step_ms), "norm_ms_min": min(norm_ms),
+        "bytes_per_param": nb + sb, "status": status, "launches_per_step": 2 * n_chunks,
+        "clocks": clocks,
+    }
+    del opt, buf
+    torch.cuda.empty_cache()
+    return res, spec
+
+
+def time_e2e(name, block, steps, warmup):
+    """Same step with the step's gradients living in pinned HOST memory: every step copies them to
+    the device (chunk by chunk, copy stream ahead of the compute stream), runs norm + step through
+    the C ABI, and reads norm and status back to the host."""
+    import torch
+    import paper_2608_11919_b200 as L
+    dev = torch.device("cuda", torch.cuda.current_device())
+    spec, buf, opt = build_workload(name, block, dev)
+    N = spec.numel
+    gbytes = buf.grad.numel() * buf.grad.element_size()
+    stage_elems = min(buf.grad.numel(), (1 << 30))                     # <= 2 GiB of pinned host memory
+    host = torch.empty(stage_elems, dtype=buf.grad.dtype, pin_memory=True)
+    host.copy_(buf.grad[:stage_elems])
+    copy_stream = torch.cuda.Stream()
+    piece = 1 << 27                                                    # 256 MiB per copy
+    result = torch.empty(2, dtype=torch.float64, pin_memory=True)
+
+    def step():
+        main = torch.cuda.current_stream()
+        copy_stream.wait_stream(main)
+        opt.t += 1
+        opt.hp.step = opt.t
+        opt.sqnorm.zero_()
+        with torch.cuda.stream(copy_stream):
+            for a in range(0, buf.grad.numel(), piece):
+                n = min(piece, buf.grad.numel() - a)
+                ha = a % stage_elems
+                if ha + n > stage_elems:
+                    ha = 0
+                buf.grad[a:a + n].copy_(host[ha:ha + n], non_blocking=True)
+        main.wait_stream(copy_stream)
+        for ch in opt.chunks:
+            L.lt_grad_sqnorm_multi(ch, opt.sqnorm, opt.workspace)
+        for ch in opt.chunks:
+            L.lt_hybrid8_step(ch, opt.block, opt.hp, opt.sqnorm, opt.status)
+        result[0:1].copy_(opt.sqnorm, non_blocking=True)
+        result[1:2].copy_(opt.status.to(torch.float64), non_blocking=True)
+
+    for _ in range(max(1, min(warmup, 3))):
+        step()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(end) / steps
+    out = {"value": N / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(gbytes), "d2h_bytes_per_step": 16,
+           "ms_per_step": ms, "what": "gradients copied from pinned host memory every step; norm + status read back"}
+    del opt, buf, host
+    torch.cuda.empty_cache()
+    return out
+
+
+def oracle_sample_time(name: str, block: int, target_params: int):
+    """Times the CPU oracle (norm + step, one thread) on the first tensors/blocks of the workload,
+    with the workload's value recipe generated on the host. Returns (params/s, sample description)."""
+    import numpy as np
+    import torch
+    import oracle as O
+    from paper_2608_11919_b200 import workloads as W
+    spec = W.SPECS[name]()
+    # sample: block-aligned head slices of the first decoder layer's tensors (embedding excluded)
+    take, left = [], target_params
+    for t, (nm, sz) in enumerate(zip(spec.names, spec.sizes)):
+        if nm == "embed" or left <= 0:
+            continue
+        n = min(sz, max(block, left // block * block))
+        take.append((t, n)); left -= n
+    stds = W.layer_stds(spec)
+    rng = np.random.default_rng(spec.seed)
+    ots = []
+    for t, n in take:
+        p = rng.normal(0, 0.02, n).astype(np.float32)
+        g = O.f32_to_bf16_bits(rng.normal(0, stds[t], n).astype(np.float32))
+        if spec.param_dtype == torch.bfloat16:
+            p = O.f32_to_bf16_bits(p)
+        ots.append(O.OracleTensor(p, g, block))
+    n_tot = sum(t.numel for t in ots)
+    hp = O.HParams(max_norm=spec.max_norm)
+    hp.step = 1
+    O.hybrid8_step(ots, block, hp, O.sqnorm(ots))            # populate the state (untimed)
+    hp.step = 2
+    t0 = time.perf_counter()
+    S = O.sqnorm(ots)
+    O.hybrid8_step(ots, block, hp, S)
+    dt = time.perf_counter() - t0
+    return n_tot / dt, f"{n_tot} params (block-aligned head slices of {len(ots)} tensors of '{name}'), 1 step, 1 thread", dt
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workloads", default="7b,3b,27b", help="first one is the headline")
+    ap.add_argument("--block", type=int, default=2048)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=128 << 20, help="params in the oracle's timed sample")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    names = [w.strip().lower() for w in args.workloads.split(",") if w.strip()]
+    head = names[0]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        from paper_2608_11919_b200 import workloads as W
+        per_step = 8 << 20          # params per reference step: keeps K + W steps within a few minutes
+        vals = []
+        for i in range(args.warmup + args.steps):
+            v, desc, dt = oracle_sample_time(head, args.block, per_step)
+            if i >= args.warmup:
+                vals.append((v, dt))
+        tot_t = sum(d for _, d in vals)
+        n_s = sum(v * d for v, d in vals)
+        value = n_s / tot_t
+        spec = W.SPECS[head]()
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_t / len(vals) * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": head, "block": args.block, "params": spec.numel,
+                           "note": "CPU oracle; each step is a bounded sample of the workload"},
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the product path)")
+    torch.cuda.set_device(local)
+    dist_on = world > 1
+    if dist_on:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peak, peak_kind = measured_peak_gbs()
+
+    results, notes = {}, {}
+    for i, name in enumerate(names if not dist_on else names[:1]):
+        try:
+            res, spec = time_resident(name, args.block, args.steps, args.warmup, rank, world, dist_on,
+                                      sample_clocks=(rank == 0))
+            results[name] = res
+        except torch.OutOfMemoryError as e:
+            torch.cuda.empty_cache()
+            notes[name] = f"skipped: out of device memory ({str(e)[:80]})"
+            if i == 0:
+                raise
+    h = results[head]
+    e2e = None
+    if not args.no_e2e:
+        e2e = time_e2e(head, args.block, max(2, min(args.steps, 5)), args.warmup)
+        if dist_on:
+            t = torch.tensor([e2e["ms_per_step"]], dtype=torch.float64, device="cuda")
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            e2e["ms_per_step"] = float(t.item())
+            e2e["value"] = h["params"] * world / (e2e["ms_per_step"] * 1e-3)
+            e2e["h2d_bytes_per_step"] *= world
+            e2e["d2h_bytes_per_step"] *= world
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, desc, dt = oracle_sample_time(head, args.block, args.cpu_sample)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+
+    if rank == 0:
+        pkey = h["param_dtype"]
+        _, sb = algorithmic_bytes_per_param(2 if pkey == "bf16" else 4, args.block)
+        traffic = STEP_TRAFFIC_BYTES_PER_PARAM.get(pkey)
+        roof = {"bound": "hbm", "kernel": "step_kernel (fused dequant/clip/AdamW/requant)",
+                "achieved": h["step_gbs"], "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": h["step_gbs"] / peak,
+                "traffic": None if traffic is None else traffic * h["params"] / h["chunks"],
+                "algorithmic_bytes_per_launch": sb * h["params"] / h["chunks"],
+                "launch_ms": h["step_ms"] / h["chunks"],
+                "whole_step_gbs": h["whole_gbs"], "whole_step_frac": h["whole_gbs"] / peak,
+                "whole_step_frac_of_8000": h["whole_gbs"] / 8000.0,
+                "norm_kernel_gbs": h["norm_gbs"], "norm_kernel_frac": h["norm_gbs"] / peak}
+        line = {"metric": METRIC, "value": h["params_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": h["ms_per_step"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": head, "params_per_gpu": h["params"], "tensors": h["tensors"],
+                           "block": args.block, "param_dtype": h["param_dtype"], "grad_dtype": "bf16",
+                           "chunks": h["chunks"], "resident_gb_per_gpu": h["resident_gb"],
+                           "l2": "inputs larger than L2 (no flush needed)",
+                           "parallelism": f"shard{world}+scalar-allreduce" if world > 1 else "single"},
+                "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": h["launches_per_step"] * args.steps, "clocks": h["clocks"],
+                "workloads": results, "notes": notes}
+        print(json.dumps(line))
+    if dist_on:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,117 @@
+/* lt.h -- C ABI of the fused global-norm clip + block-wise 8-bit AdamW optimizer step (sm_100a).
+ *
+ * The operator is the optimizer-side component of the paper's Sec. 3.5 ("Hybrid 8-bit operator"):
+ * Adam moments held as 8-bit codes with block-wise scales, updated by an AdamW step, coupled with a
+ * fast global-norm gradient clip. Here every step of it runs on the GPU, on the caller's stream.
+ *
+ * Conventions for every function
+ *   - returns LT_OK (0) or a negative lt_status; never throws, never aborts, never synchronises the
+ *     stream (one exception: the FIRST call on a device uploads the code tables and waits for that
+ *     upload; make that call before any stream capture);
+ *   - never allocates or frees device memory;
+ *   - lt_tensor arrays, lt_hparams and out-parameters of the host-side queries are HOST memory read
+ *     during the call; every pointer INSIDE an lt_tensor, and d_sqnorm / d_status / d_workspace, are
+ *     DEVICE pointers owned by the caller that must stay valid until the enqueued work has run;
+ *   - arguments are validated on the host before anything is launched: a call that returns an
+ *     error has enqueued nothing (LT_ERR_CUDA excepted: a launch itself failed).
+ *
+ * Data layout. A tensor is a flat array of `numel` elements. Its 8-bit state is one byte per element
+ * per moment (m_code: index into the signed 256-entry map; v_code: index into the unsigned map) and
+ * one fp32 scale per block of `block` consecutive elements per moment (the block's absolute maximum).
+ * Blocks restart at every tensor; the last block of a tensor may be short. The value-zero state is
+ * m_code = 127, v_code = 0, scales = 0.
+ */
+#ifndef LT_H_
+#define LT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LT_OK = 0,
+    LT_ERR_INVALID_ARG = -1,  /* null pointer, negative size, bad enum, bad hyper-parameter */
+    LT_ERR_ALIGNMENT = -2,    /* a pointer is not aligned to its element size */
+    LT_ERR_UNSUPPORTED = -3,  /* block size not a power of two in [256, 16384] */
+    LT_ERR_CUDA = -4,         /* a CUDA call or launch failed (the CUDA error is consumed) */
+    LT_ERR_WORKSPACE = -5     /* workspace missing, misaligned or smaller than lt_workspace_bytes() */
+} lt_status;
+
+typedef enum { LT_F32 = 0, LT_BF16 = 1 } lt_dtype;
+
+/* A CUDA stream handle (cudaStream_t / CUstream); NULL is the default stream. */
+typedef struct CUstream_st* lt_stream;
+
+typedef struct {
+    void* param;          /* device [numel] of param_dtype; read and written by lt_hybrid8_step      */
+    const void* grad;     /* device [numel] of grad_dtype; read only, never rescaled in place        */
+    uint8_t* m_code;      /* device [numel]                                                         */
+    uint8_t* v_code;      /* device [numel]                                                         */
+    float* m_absmax;      /* device [ceil(numel / block)]                                           */
+    float* v_absmax;      /* device [ceil(numel / block)]                                           */
+    int64_t numel;        /* >= 0; a tensor with 0 elements is skipped                               */
+    int32_t param_dtype;  /* lt_dtype                                                               */
+    int32_t grad_dtype;   /* lt_dtype                                                               */
+} lt_tensor;
+
+/* Hyper-parameters of one optimizer step (the paper's training-configuration table uses
+ * beta1 0.9, beta2 0.999, eps 1e-8, lr 1e-5, weight_decay 0.01, max_norm 1.0). `step` is the 1-based
+ * step count, supplied by the caller. max_norm <= 0 or +inf disables clipping. */
+typedef struct {
+    float lr, beta1, beta2, eps, weight_decay, max_norm;
+    int64_t step;
+} lt_hparams;
+
+/* Bytes of 8-bit state for a tensor of `numel` elements: codes per moment (= numel) and scales per
+ * moment (= 4 * ceil(numel / block)). The paper's optimizer-memory rows (full 8-bit vs 2 % 8-bit
+ * Adam states, solver-snapshot table) are consistent with exactly this footprint at block 4096. */
+int lt_hybrid8_state_bytes(int64_t numel, int32_t block, int64_t* code_bytes, int64_t* absmax_bytes);
+
+/* Copies the 256-entry code map (signed: first moment, unsigned: second moment) to host memory.
+ * Decade e = 0..6 with scale 10^(e-6) holds 2^e (signed) or 2^(e+1) (unsigned) cell mid-points of a
+ * uniform grid on [0.1, 1]; plus 0.0 and +1.0 (the paper names only a "CPU 8-bit AdamW format", Sec.
+ * 3.5; this map is this library's reading of it). */
+int lt_hybrid8_code_table(int32_t is_signed, float* out256);
+
+/* Size in bytes of the device scratch lt_grad_sqnorm_multi needs (a constant, a few KB). The scratch
+ * must be 256-byte aligned; its contents need no initialisation and mean nothing between calls.
+ * Calls that run concurrently on the GPU must not share one scratch buffer. */
+int64_t lt_workspace_bytes(void);
+
+/* S0 -- puts the 8-bit state of every tensor to value zero (m_code 127, v_code 0, scales 0).
+ * Uses m_code, v_code, m_absmax, v_absmax, numel. (Sec. 3.5: moments "in CPU 8-bit AdamW format".) */
+int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt_stream stream);
+
+/* S1 -- multi-tensor squared L2 norm (Sec. 3.5: the clip "computes per-tensor norms ... aggregates
+ * the global norm"). ADDS sum_t sum_i grad[t][i]^2 to *d_sqnorm (device double). The caller zeroes
+ * *d_sqnorm before the first chunk of an optimizer step and may call this once per chunk of the
+ * tensor list. Uses grad, grad_dtype, numel. Accumulation is fp64 over exact fp32 squares; the
+ * result is bit-reproducible for a given tensor list on a given device. */
+int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
+                         void* d_workspace, int64_t workspace_bytes, lt_stream stream);
+
+/* S2..S5 -- the fused step (Sec. 3.5: dequantize, "8-bit state updates", requantize with
+ * "block-wise scale handling", under the clip's single scale). Reads S = *d_sqnorm, the squared norm
+ * over ALL gradients of this optimizer step (the tensor list may be one chunk of them):
+ *     c   = min(1, max_norm / (sqrt(S) + 1e-6))                       (1 if clipping is disabled)
+ *     g   = c * grad;   m = QS[m_code] * m_absmax[b];   v = QU[v_code] * v_absmax[b]
+ *     m'  = beta1 m + (1 - beta1) g;    v' = beta2 v + (1 - beta2) g^2
+ *     p  <- p (1 - lr wd) - lr / (1 - beta1^t) * m' / (sqrt(v') / sqrt(1 - beta2^t) + eps)
+ *     per block: m_absmax = max |m'|, v_absmax = max v', codes = nearest map entry of m'/m_absmax,
+ *     v'/v_absmax (ties to the lower index; an all-zero block gets zero codes and scale 0).
+ * If S is NaN or Inf nothing is written except bit 0 of *d_status (the paper's "non-finite gradients
+ * are skipped", training-configuration table); the caller clears d_status when it wants to.
+ * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
+ * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). */
+int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
+                    const double* d_sqnorm, int32_t* d_status, lt_stream stream);
+
+/* Name of a status code (static string). */
+const char* lt_status_str(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LT_H_ */

@@ -1,0 +1,276 @@
+// Host side of the C ABI: argument validation, code-map construction, per-launch descriptor packing.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "lt_common.cuh"
+
+namespace lt {
+
+// ---- code maps (host) --------------------------------------------------------------------------
+// Signed map: 127 negative magnitudes (descending), 0.0, 127 positive magnitudes, +1.0.
+// Unsigned map: 0.0, 254 magnitudes, +1.0. Magnitudes of decade e: 10^(e-6) * (0.1 + 0.9 (j+.5)/n_e),
+// n_e = 2^e (signed) or 2^(e+1) (unsigned), formed in double and rounded once to fp32.
+struct HostTables {
+    float qs[256], qu[256];
+    float mid_s[256], mid_u[256];   // [k] = (T[k] + T[k+1]) / 2 rounded toward -inf; [255] = +inf
+    HostTables() {
+        static const double decade[7] = {1e-6, 1e-5, 1e-4, 1e-3, 1e-2, 1e-1, 1e0};
+        int is = 0, iu = 1;
+        qu[0] = 0.0f;
+        qs[127] = 0.0f;
+        for (int e = 0; e < 7; ++e) {
+            const int ns = 1 << e, nu = 2 << e;
+            for (int j = 0; j < ns; ++j) {
+                const float f = (float)(decade[e] * (0.1 + 0.9 * ((double)j + 0.5) / (double)ns));
+                qs[128 + is] = f;
+                qs[126 - is] = -f;
+                ++is;
+            }
+            for (int j = 0; j < nu; ++j)
+                qu[iu++] = (float)(decade[e] * (0.1 + 0.9 * ((double)j + 0.5) / (double)nu));
+        }
+        qs[255] = 1.0f;
+        qu[255] = 1.0f;
+        fill_mid(qs, mid_s);
+        fill_mid(qu, mid_u);
+    }
+    // For fp32 x and a mid-point M that is exact in double: x > M  <=>  x > round_down(M).
+    static void fill_mid(const float* T, float* mid) {
+        for (int k = 0; k < 255; ++k) {
+            const double m = ((double)T[k] + (double)T[k + 1]) * 0.5;
+            float f = (float)m;
+            if ((double)f > m) f = std::nextafterf(f, -INFINITY);
+            mid[k] = f;
+        }
+        mid[255] = INFINITY;
+    }
+};
+
+static const HostTables& host_tables() {
+    static HostTables t;
+    return t;
+}
+const float* host_table(bool is_signed) { return is_signed ? host_tables().qs : host_tables().qu; }
+const float* host_mid_rd(bool is_signed) { return is_signed ? host_tables().mid_s : host_tables().mid_u; }
+
+// ---- per-device set-up ---------------------------------------------------------------------------
+static std::mutex g_mu;
+static DeviceInfo g_dev[64];
+
+int ensure_device(cudaStream_t stream, DeviceInfo** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LT_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceInfo& d = g_dev[dev];
+    if (!d.tables_ready) {
+        if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            d.sm_count <= 0) { cudaGetLastError(); return LT_ERR_CUDA; }
+        if (upload_tables(stream) != LT_OK) return LT_ERR_CUDA;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
+        d.tables_ready = true;
+    }
+    *out = &d;
+    return LT_OK;
+}
+
+static bool valid_block(int32_t block) {
+    return block >= 256 && block <= 16384 && (block & (block - 1)) == 0;
+}
+static bool valid_dtype(int32_t d) { return d == LT_F32 || d == LT_BF16; }
+static int esize(int32_t d) { return d == LT_F32 ? 4 : 2; }
+static bool aligned(const void* p, int a) { return ((uintptr_t)p % (uintptr_t)a) == 0; }
+
+// which fields a call needs
+enum { NEED_GRAD = 1, NEED_PARAM = 2, NEED_STATE = 4 };
+
+static int validate_tensors(const lt_tensor* t, int32_t n, int need) {
+    if (n < 0 || (n > 0 && t == nullptr)) return LT_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < n; ++i) {
+        const lt_tensor& x = t[i];
+        if (x.numel < 0) return LT_ERR_INVALID_ARG;
+        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;   // keeps per-launch block counts in int32
+        if (x.numel == 0) continue;
+        if (need & NEED_GRAD) {
+            if (!valid_dtype(x.grad_dtype) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
+            if (!aligned(x.grad, esize(x.grad_dtype))) return LT_ERR_ALIGNMENT;
+        }
+        if (need & NEED_PARAM) {
+            if (!valid_dtype(x.param_dtype) || x.param == nullptr) return LT_ERR_INVALID_ARG;
+            if (!aligned(x.param, esize(x.param_dtype))) return LT_ERR_ALIGNMENT;
+        }
+        if (need & NEED_STATE) {
+            if (!x.m_code || !x.v_code || !x.m_absmax || !x.v_absmax) return LT_ERR_INVALID_ARG;
+            if (!aligned(x.m_absmax, 4) || !aligned(x.v_absmax, 4)) return LT_ERR_ALIGNMENT;
+        }
+    }
+    return LT_OK;
+}
+
+// Packs tensors [*i, ...) into one launch's descriptors; advances *i.
+static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, StepParams* P, bool with_pg) {
+    int cnt = 0;
+    int64_t blocks = 0;
+    while (*i < n && cnt < kCap) {
+        const lt_tensor& x = t[*i];
+        if (x.numel == 0) { ++*i; continue; }
+        const int64_t nb = (x.numel + block - 1) / block;
+        if (blocks + nb > 0x7fffffff) break;   // next launch; one tensor alone always fits (numel <= 2^38)
+        StepDesc& d = P->t[cnt];
+        d.p = with_pg ? x.param : nullptr;
+        d.g = with_pg ? x.grad : nullptr;
+        d.mc = x.m_code; d.vc = x.v_code; d.am = x.m_absmax; d.av = x.v_absmax;
+        d.numel = x.numel;
+        blocks += nb;
+        d.blk_end = (int32_t)blocks;
+        int flags = 0;
+        bool vec = aligned(x.m_code, 4) && aligned(x.v_code, 4);
+        if (with_pg) {
+            if (x.param_dtype == LT_BF16) flags |= kFlagParamBf16;
+            if (x.grad_dtype == LT_F32) flags |= kFlagGradF32;
+            vec = vec && aligned(x.param, 4 * esize(x.param_dtype)) && aligned(x.grad, 4 * esize(x.grad_dtype));
+        }
+        if (vec) flags |= kFlagVecOk;
+        d.flags = flags;
+        ++cnt; ++*i;
+    }
+    P->n = cnt;
+    P->total_blocks = (int32_t)blocks;
+}
+
+}  // namespace lt
+
+using namespace lt;
+
+extern "C" {
+
+const char* lt_status_str(int status) {
+    switch (status) {
+        case LT_OK: return "LT_OK";
+        case LT_ERR_INVALID_ARG: return "LT_ERR_INVALID_ARG";
+        case LT_ERR_ALIGNMENT: return "LT_ERR_ALIGNMENT";
+        case LT_ERR_UNSUPPORTED: return "LT_ERR_UNSUPPORTED";
+        case LT_ERR_CUDA: return "LT_ERR_CUDA";
+        case LT_ERR_WORKSPACE: return "LT_ERR_WORKSPACE";
+        default: return "LT_ERR_UNKNOWN";
+    }
+}
+
+int lt_hybrid8_state_bytes(int64_t numel, int32_t block, int64_t* code_bytes, int64_t* absmax_bytes) {
+    if (numel < 0 || !code_bytes || !absmax_bytes) return LT_ERR_INVALID_ARG;
+    if (!valid_block(block)) return LT_ERR_UNSUPPORTED;
+    *code_bytes = numel;
+    *absmax_bytes = 4 * ((numel + block - 1) / block);
+    return LT_OK;
+}
+
+int lt_hybrid8_code_table(int32_t is_signed, float* out256) {
+    if (!out256) return LT_ERR_INVALID_ARG;
+    std::memcpy(out256, host_table(is_signed != 0), 256 * sizeof(float));
+    return LT_OK;
+}
+
+int64_t lt_workspace_bytes(void) { return kWorkspaceBytes; }
+
+int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt_stream stream) {
+    if (!valid_block(block)) return LT_ERR_UNSUPPORTED;
+    int rc = validate_tensors(tensors, n, NEED_STATE);
+    if (rc != LT_OK) return rc;
+    DeviceInfo* dev = nullptr;
+    if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
+    StepParams P;
+    std::memset(&P.s, 0, sizeof(P.s));
+    P.sqnorm = nullptr; P.status = nullptr;
+    int32_t i = 0;
+    while (i < n) {
+        pack_step(tensors, n, block, &i, &P, false);
+        if (P.n == 0) continue;
+        if ((rc = launch_state_init(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+    }
+    return LT_OK;
+}
+
+int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
+                         void* d_workspace, int64_t workspace_bytes, lt_stream stream) {
+    int rc = validate_tensors(tensors, n, NEED_GRAD);
+    if (rc != LT_OK) return rc;
+    if (!d_sqnorm) return LT_ERR_INVALID_ARG;
+    if (!aligned(d_sqnorm, 8)) return LT_ERR_ALIGNMENT;
+    if (!d_workspace || workspace_bytes < kWorkspaceBytes || !aligned(d_workspace, 256)) return LT_ERR_WORKSPACE;
+    DeviceInfo* dev = nullptr;
+    if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
+
+    NormParams P;
+    P.ticket = (unsigned int*)d_workspace;
+    P.partials = (double*)((char*)d_workspace + 256);
+    P.out = d_sqnorm;
+    int32_t i = 0;
+    while (i < n) {
+        int cnt = 0;
+        int64_t items = 0;
+        while (i < n && cnt < kCap) {
+            const lt_tensor& x = tensors[i];
+            if (x.numel == 0) { ++i; continue; }
+            const uintptr_t a = (uintptr_t)x.grad;
+            const int lead = (int)(a & 15);
+            const int64_t span = lead + x.numel * esize(x.grad_dtype);
+            const int64_t it = (span + kNormItemBytes - 1) / kNormItemBytes;
+            if (items + it > 0x7fffffff) break;
+            NormDesc& d = P.t[cnt];
+            d.base16 = (const void*)(a - lead);
+            d.span_bytes = span;
+            items += it;
+            d.item_end = (int32_t)items;
+            d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
+            ++cnt; ++i;
+        }
+        if (cnt == 0) continue;
+        P.n = cnt;
+        P.total_items = (int32_t)items;
+        // the arrival counter must start at zero whatever an earlier (possibly failed) launch left
+        if (cudaMemsetAsync(P.ticket, 0, 256, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
+        if ((rc = launch_sqnorm(P, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+    }
+    return LT_OK;
+}
+
+int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
+                    const double* d_sqnorm, int32_t* d_status, lt_stream stream) {
+    if (!valid_block(block)) return LT_ERR_UNSUPPORTED;
+    if (!hp) return LT_ERR_INVALID_ARG;
+    int rc = validate_tensors(tensors, n, NEED_GRAD | NEED_PARAM | NEED_STATE);
+    if (rc != LT_OK) return rc;
+    if (hp->step < 1 || !(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) ||
+        !(hp->eps >= 0.0f) || !std::isfinite(hp->lr) || !std::isfinite(hp->weight_decay) || std::isnan(hp->max_norm))
+        return LT_ERR_INVALID_ARG;
+    const bool clip_on = hp->max_norm > 0.0f && !std::isinf(hp->max_norm);
+    if (clip_on && !d_sqnorm) return LT_ERR_INVALID_ARG;
+    if (d_sqnorm && !aligned(d_sqnorm, 8)) return LT_ERR_ALIGNMENT;
+    if (d_status && !aligned(d_status, 4)) return LT_ERR_ALIGNMENT;
+    DeviceInfo* dev = nullptr;
+    if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
+
+    StepParams P;
+    // per-step scalars: formed in double, rounded once to fp32
+    const double b1 = (double)hp->beta1, b2 = (double)hp->beta2, t = (double)hp->step;
+    const double bc1 = 1.0 - std::pow(b1, t), bc2 = 1.0 - std::pow(b2, t);
+    P.s.beta1 = hp->beta1; P.s.beta2 = hp->beta2;
+    P.s.omb1 = (float)(1.0 - b1); P.s.omb2 = (float)(1.0 - b2);
+    P.s.step_size = (float)((double)hp->lr / bc1);
+    P.s.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
+    P.s.decay = (float)(1.0 - (double)hp->lr * (double)hp->weight_decay);
+    P.s.eps = hp->eps;
+    P.s.max_norm = hp->max_norm;
+    P.s.clip_on = clip_on ? 1 : 0;
+    P.sqnorm = d_sqnorm;
+    P.status = d_status;
+    int32_t i = 0;
+    while (i < n) {
+        pack_step(tensors, n, block, &i, &P, true);
+        if (P.n == 0) continue;
+        if ((rc = launch_step(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+    }
+    return LT_OK;
+}
+
+}  // extern "C"

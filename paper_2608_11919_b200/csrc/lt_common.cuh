@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of liblt_hybrid8 (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lt.h"
+
+namespace lt {
+
+// Tensors per launch: descriptors travel as kernel parameters (no device table, no copy to keep
+// alive), and the parameter space of sm_100 holds 32764 bytes.
+constexpr int kCap = 480;
+
+constexpr int kFlagParamBf16 = 1;
+constexpr int kFlagGradF32 = 2;
+constexpr int kFlagVecOk = 4;   // every pointer allows 4-element vector access
+
+struct StepDesc {               // 64 bytes
+    void* p;
+    const void* g;
+    uint8_t* mc;
+    uint8_t* vc;
+    float* am;
+    float* av;
+    int64_t numel;
+    int32_t blk_end;            // exclusive end of this tensor's range of launch-wide block indices
+    int32_t flags;
+};
+
+struct StepScalars {
+    float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, decay, eps, max_norm;
+    int32_t clip_on;
+};
+
+struct StepParams {
+    StepDesc t[kCap];
+    StepScalars s;
+    const double* sqnorm;
+    int32_t* status;
+    int32_t n;
+    int32_t total_blocks;
+};
+
+struct NormDesc {               // 24 bytes
+    const void* base16;         // gradient address rounded down to 16 bytes
+    int64_t span_bytes;         // lead bytes + numel * element size
+    int32_t item_end;           // exclusive end of this tensor's range of launch-wide work items
+    int32_t lead_f32;           // lead bytes (0..15) | grad_is_f32 << 8
+};
+
+struct NormParams {
+    NormDesc t[kCap];
+    double* partials;           // workspace: one double per CTA
+    unsigned int* ticket;       // workspace: arrival counter, zero between launches
+    double* out;                // *out += total
+    int32_t n;
+    int32_t total_items;
+};
+
+struct DeviceInfo {
+    int sm_count = 0;
+    bool tables_ready = false;
+};
+
+// per-device lazy set-up (SM count, code tables in constant memory). Returns LT_OK or LT_ERR_CUDA.
+int ensure_device(cudaStream_t stream, DeviceInfo** out);
+
+// host copies of the code maps and of the search thresholds (mid-points rounded toward -inf)
+const float* host_table(bool is_signed);
+const float* host_mid_rd(bool is_signed);
+
+int launch_state_init(const StepParams& p, int block, int sm_count, cudaStream_t s);
+int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
+int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
+int upload_tables(cudaStream_t s);
+
+constexpr int kNormThreads = 512;
+constexpr int kNormVecPerThread = 4;
+constexpr int kNormItemBytes = kNormThreads * kNormVecPerThread * 16;
+constexpr int kNormMaxCtas = 1024;
+constexpr int64_t kWorkspaceBytes = 256 + kNormMaxCtas * 8;
+
+}  // namespace lt

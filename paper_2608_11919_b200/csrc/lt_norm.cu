@@ -1,0 +1,145 @@
+// S1: multi-tensor squared L2 norm of the gradients, finished on the device.
+//
+// Bound: HBM read bandwidth, 2 bytes per bf16 gradient element, read once. A work item is 32 KiB of
+// one tensor's 16-byte-aligned span; a CTA of 512 threads issues four independent 16-byte streaming
+// loads per thread per item and the grid is a whole number of CTAs per SM, walking items in a
+// grid-stride loop, so each SM keeps 64 KiB of loads in flight.
+//
+// Accuracy and reproducibility. Each thread converts its bf16 values to fp64 (exact), and adds their
+// exact squares to an fp64 accumulator with one fused multiply-add each, so only the running fp64
+// sum rounds. Per-CTA fp64 partials go to the workspace; the last CTA to arrive
+// (an atomic ticket, not a wait) adds them in index order and accumulates the launch total into
+// *out. Nothing depends on arrival order, so the result is bit-reproducible.
+#include "lt_common.cuh"
+
+namespace lt {
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// eight squares of one vector of bf16 added to an fp64 accumulator. A bf16 value converts to fp64
+// exactly and its square has 16 significant bits, so every product is exact and only the running
+// sum rounds (in fp64). (Summing the squares in fp32 first is biased: the addends have few
+// significant bits, ties are frequent, and ties-to-even then always rounds the sum down.)
+__device__ __forceinline__ double sq8_bf16(const uint4& v, double acc) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const double lo = (double)bf16_lo(w[i]), hi = (double)bf16_hi(w[i]);
+        acc = fma(lo, lo, acc);
+        acc = fma(hi, hi, acc);
+    }
+    return acc;
+}
+
+__device__ __forceinline__ double sq4_f32(const uint4& v) {
+    const double a = (double)__uint_as_float(v.x), b = (double)__uint_as_float(v.y);
+    const double c = (double)__uint_as_float(v.z), d = (double)__uint_as_float(v.w);
+    return (a * a + b * b) + (c * c + d * d);
+}
+
+// elements of a vector that straddles the tensor's first or last byte, read one by one
+__device__ __forceinline__ double sq_partial(const char* base, int64_t off, int64_t lo, int64_t hi, bool f32) {
+    double acc = 0.0;
+    if (f32) {
+        for (int j = 0; j < 4; ++j) {
+            const int64_t b = off + 4 * j;
+            if (b >= lo && b + 4 <= hi) { const double x = (double)*(const float*)(base + b); acc += x * x; }
+        }
+    } else {
+        for (int j = 0; j < 8; ++j) {
+            const int64_t b = off + 2 * j;
+            if (b >= lo && b + 2 <= hi) {
+                const double x = (double)__uint_as_float((uint32_t)*(const unsigned short*)(base + b) << 16);
+                acc += x * x;
+            }
+        }
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(kNormThreads, 2) sqnorm_kernel(const __grid_constant__ NormParams P) {
+    __shared__ double s_warp[kNormThreads / 32];
+    __shared__ bool s_last;
+    const int tid = threadIdx.x;
+    double acc = 0.0;
+    int t = 0;
+    int item_begin = 0;
+    for (int w = blockIdx.x; w < P.total_items; w += gridDim.x) {
+        while (w >= P.t[t].item_end) { item_begin = P.t[t].item_end; ++t; }
+        const NormDesc& d = P.t[t];
+        const char* base = (const char*)d.base16;
+        const int64_t lo = d.lead_f32 & 0xff;
+        const bool f32 = (d.lead_f32 >> 8) != 0;
+        const int64_t hi = d.span_bytes;
+        const int64_t item_off = (int64_t)(w - item_begin) * kNormItemBytes;
+        if (item_off >= lo && item_off + kNormItemBytes <= hi) {
+            uint4 v[kNormVecPerThread];
+#pragma unroll
+            for (int k = 0; k < kNormVecPerThread; ++k)
+                v[k] = ld_stream16(base + item_off + (int64_t)(k * kNormThreads + tid) * 16);
+            if (!f32) {
+#pragma unroll
+                for (int k = 0; k < kNormVecPerThread; ++k) acc = sq8_bf16(v[k], acc);
+            } else {
+#pragma unroll
+                for (int k = 0; k < kNormVecPerThread; ++k) acc += sq4_f32(v[k]);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < kNormVecPerThread; ++k) {
+                const int64_t off = item_off + (int64_t)(k * kNormThreads + tid) * 16;
+                if (off >= lo && off + 16 <= hi) {
+                    const uint4 v = ld_stream16(base + off);
+                    acc = f32 ? acc + sq4_f32(v) : sq8_bf16(v, acc);
+                } else if (off + 16 > lo && off < hi) {
+                    acc += sq_partial(base, off, lo, hi, f32);
+                }
+            }
+        }
+    }
+    // CTA reduction in a fixed order
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((tid & 31) == 0) s_warp[tid >> 5] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        double s = 0.0;
+        for (int i = 0; i < kNormThreads / 32; ++i) s += s_warp[i];
+        P.partials[blockIdx.x] = s;
+        __threadfence();
+        const unsigned int ticket = atomicAdd(P.ticket, 1u);
+        s_last = (ticket == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (s_last && tid < 32) {
+        __threadfence();
+        // lanes take partials i = lane, lane + 32, ... in order, then a fixed shuffle tree
+        double s = 0.0;
+        for (int i = tid; i < (int)gridDim.x; i += 32) s += __ldcg(&P.partials[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (tid == 0) {
+            *P.out = *P.out + s;
+            *P.ticket = 0u;
+        }
+    }
+}
+
+int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s) {
+    int grid = 2 * sm_count;
+    if (grid > kNormMaxCtas) grid = kNormMaxCtas;
+    if (grid > p.total_items) grid = p.total_items;
+    if (grid < 1) grid = 1;
+    sqnorm_kernel<<<grid, kNormThreads, 0, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return LT_ERR_CUDA;
+    return LT_OK;
+}
+
+}  // namespace lt
