@@ -14,6 +14,9 @@ namespace lt {
 struct HostTables {
     float qs[256], qu[256];
     float mid_s[256], mid_u[256];   // [k] = (T[k] + T[k+1]) / 2 rounded toward -inf; [255] = +inf
+    QuantLut lut_u[kLutEntries];    // see build_lut
+    QuantLut lut_s[kLutEntries];
+    bool lut_ok;
     HostTables() {
         static const double decade[7] = {1e-6, 1e-5, 1e-4, 1e-3, 1e-2, 1e-1, 1e0};
         int is = 0, iu = 1;
@@ -34,6 +37,37 @@ struct HostTables {
         qu[255] = 1.0f;
         fill_mid(qs, mid_s);
         fill_mid(qu, mid_u);
+        lut_ok = build_lut(mid_u, 7, false, lut_u) && build_lut(mid_s, 6, true, lut_s);
+    }
+    static int code_of(const float* mid, float x) {   // number of thresholds strictly below x
+        int c = 0;
+        for (int k = 0; k < 255; ++k) c += (x > mid[k]) ? 1 : 0;
+        return c;
+    }
+    static float from_bits(uint32_t b) { float f; std::memcpy(&f, &b, 4); return f; }
+    // Direct-lookup form of the search. A bucket is the set of floats that share sign, exponent field
+    // (96..127, i.e. magnitude in [2^-31, 2)) and the top `mbits` mantissa bits. The code map is so
+    // coarse against that grid that a bucket holds at most one threshold; its entry is that threshold
+    // (or +inf) and the code below it: code(x) = base + (x > threshold). Unsigned map: 32 x 128
+    // buckets. Signed map: 32 x 64 buckets of the magnitude, positive half first, negative half second.
+    static bool build_lut(const float* mid, int mbits, bool is_signed, QuantLut* lut) {
+        const int per_binade = 1 << mbits, half = 32 * per_binade;
+        for (int h = 0; h < (is_signed ? 2 : 1); ++h) {
+            for (int key = 0; key < half; ++key) {
+                const uint32_t lo = ((uint32_t)(96 + key / per_binade) << 23) |
+                                    ((uint32_t)(key % per_binade) << (23 - mbits));
+                const uint32_t hi = lo | ((1u << (23 - mbits)) - 1u);
+                const float xa = h == 0 ? from_bits(lo) : -from_bits(hi);   // smallest value of the bucket
+                const float xb = h == 0 ? from_bits(hi) : -from_bits(lo);   // largest
+                const int ca = code_of(mid, xa), cb = code_of(mid, xb);
+                QuantLut& e = lut[h * half + key];
+                e.base = ca;
+                if (cb == ca) e.threshold = INFINITY;
+                else if (cb == ca + 1) e.threshold = mid[ca];
+                else return false;
+            }
+        }
+        return true;
     }
     // For fp32 x and a mid-point M that is exact in double: x > M  <=>  x > round_down(M).
     static void fill_mid(const float* T, float* mid) {
@@ -53,6 +87,10 @@ static const HostTables& host_tables() {
 }
 const float* host_table(bool is_signed) { return is_signed ? host_tables().qs : host_tables().qu; }
 const float* host_mid_rd(bool is_signed) { return is_signed ? host_tables().mid_s : host_tables().mid_u; }
+const QuantLut* host_lut(bool is_signed) {
+    if (!host_tables().lut_ok) return nullptr;
+    return is_signed ? host_tables().lut_s : host_tables().lut_u;
+}
 
 // ---- per-device set-up ---------------------------------------------------------------------------
 static std::mutex g_mu;
@@ -262,6 +300,8 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
     P.s.eps = hp->eps;
     P.s.max_norm = hp->max_norm;
     P.s.clip_on = clip_on ? 1 : 0;
+    // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps
+    P.s.precise_param = (hp->eps < 1e-15f) ? 1 : 0;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
     int32_t i = 0;

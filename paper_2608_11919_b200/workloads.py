@@ -130,7 +130,20 @@ def scaled_decoder_spec(name: str, hidden: int, layers: int, q_heads: int, kv_he
                     seed=seed, grad_std=grad_std, grad_kind=grad_kind, max_norm=1.0, steps=1)
 
 
-SPECS = {"tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
+def small_spec() -> Spec:
+    """About 0.5 B parameters (4 GB resident, well above L2): a 3B-like list with 6 layers and a
+    32768-row embedding; the case profiler captures run on."""
+    return _decoder("small", 2048, 6, 16, 2, 11008, 32768, True, param_dtype=torch.float32, seed=5,
+                    grad_std=1e-4, grad_kind="layer_normal", max_norm=1.0, steps=1)
+
+
+def small_bf16_spec() -> Spec:
+    s = small_spec()
+    s.name, s.param_dtype, s.seed = "small_bf16", torch.bfloat16, 6
+    return s
+
+
+SPECS = {"small": small_spec, "small_bf16": small_bf16_spec, "tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
 
 
 def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:
