@@ -14,8 +14,8 @@ namespace lt {
 struct HostTables {
     float qs[256], qu[256];
     float mid_s[256], mid_u[256];   // [k] = (T[k] + T[k+1]) / 2 rounded toward -inf; [255] = +inf
-    QuantLut lut_u[kLutEntries];    // see build_lut
-    QuantLut lut_s[kLutEntries];
+    uint32_t lut_u[kLutEntries];    // see build_lut
+    uint32_t lut_s[kLutEntries];
     bool lut_ok;
     HostTables() {
         static const double decade[7] = {1e-6, 1e-5, 1e-4, 1e-3, 1e-2, 1e-1, 1e0};
@@ -46,25 +46,43 @@ struct HostTables {
     }
     static float from_bits(uint32_t b) { float f; std::memcpy(&f, &b, 4); return f; }
     // Direct-lookup form of the search. A bucket is the set of floats that share sign, exponent field
-    // (96..127, i.e. magnitude in [2^-31, 2)) and the top `mbits` mantissa bits. The code map is so
-    // coarse against that grid that a bucket holds at most one threshold; its entry is that threshold
-    // (or +inf) and the code below it: code(x) = base + (x > threshold). Unsigned map: 32 x 128
-    // buckets. Signed map: 32 x 64 buckets of the magnitude, positive half first, negative half second.
-    static bool build_lut(const float* mid, int mbits, bool is_signed, QuantLut* lut) {
-        const int per_binade = 1 << mbits, half = 32 * per_binade;
+    // (96..127, i.e. magnitude in [2^-31, 2)) and the top `mbits` mantissa bits; `frac` is the rest of
+    // the mantissa (fbits = 23 - mbits bits). The code map is so coarse against that grid that a
+    // bucket holds at most one threshold T, so code(x) = base + (x > T) with base = code of the
+    // bucket's smallest value. An entry packs both into one word so that ONE integer add decides:
+    //   x >= 0:  entry = base << 24 | (0xFFFFFF - frac(T));   code = (entry + frac(x)) >> 24
+    //            (the add carries into bits 24.. exactly when frac(x) > frac(T); no T: frac(T) = all ones)
+    //   x <  0:  entry = (base + 1) << 24 | frac(T);          code = (entry + ~frac(x)) >> 24
+    //            (= entry - frac(x) - 1, which keeps base + 1 exactly when frac(x) < frac(T), i.e. x > T;
+    //            no T: frac(T) = 0)
+    // Unsigned map: 32 x 128 buckets. Signed map: 32 x 64 buckets of the magnitude, positive half
+    // first, negative half second.
+    static bool build_lut(const float* mid, int mbits, bool is_signed, uint32_t* lut) {
+        const int per_binade = 1 << mbits, half = 32 * per_binade, fbits = 23 - mbits;
+        const uint32_t fmask = (1u << fbits) - 1u;
         for (int h = 0; h < (is_signed ? 2 : 1); ++h) {
             for (int key = 0; key < half; ++key) {
                 const uint32_t lo = ((uint32_t)(96 + key / per_binade) << 23) |
-                                    ((uint32_t)(key % per_binade) << (23 - mbits));
-                const uint32_t hi = lo | ((1u << (23 - mbits)) - 1u);
+                                    ((uint32_t)(key % per_binade) << fbits);
+                const uint32_t hi = lo | fmask;
                 const float xa = h == 0 ? from_bits(lo) : -from_bits(hi);   // smallest value of the bucket
                 const float xb = h == 0 ? from_bits(hi) : -from_bits(lo);   // largest
                 const int ca = code_of(mid, xa), cb = code_of(mid, xb);
-                QuantLut& e = lut[h * half + key];
-                e.base = ca;
-                if (cb == ca) e.threshold = INFINITY;
-                else if (cb == ca + 1) e.threshold = mid[ca];
-                else return false;
+                bool has_t = false;
+                uint32_t tf = 0;
+                if (cb == ca + 1) {
+                    uint32_t tb; std::memcpy(&tb, &mid[ca], 4);
+                    if (((tb & 0x7fffffffu) & ~fmask) != lo) return false;   // T must lie in this bucket
+                    has_t = true;
+                    tf = tb & fmask;
+                } else if (cb != ca) {
+                    return false;
+                }
+                uint32_t e;
+                if (h == 0) e = ((uint32_t)ca << 24) | (0xFFFFFFu - (has_t ? tf : fmask));
+                else e = ((uint32_t)(ca + 1) << 24) | (has_t ? tf : 0u);
+                if (h == 1 && ca + 1 > 255) return false;
+                lut[h * half + key] = e;
             }
         }
         return true;
@@ -87,7 +105,7 @@ static const HostTables& host_tables() {
 }
 const float* host_table(bool is_signed) { return is_signed ? host_tables().qs : host_tables().qu; }
 const float* host_mid_rd(bool is_signed) { return is_signed ? host_tables().mid_s : host_tables().mid_u; }
-const QuantLut* host_lut(bool is_signed) {
+const uint32_t* host_lut(bool is_signed) {
     if (!host_tables().lut_ok) return nullptr;
     return is_signed ? host_tables().lut_s : host_tables().lut_u;
 }

@@ -34,11 +34,7 @@ struct StepScalars {
     int32_t precise_param;      // 1: IEEE sqrt and divide in the parameter update (tiny eps)
 };
 
-// One bucket of the direct-lookup quantizer: code(x) = base + (x > threshold).
-struct QuantLut {
-    float threshold;
-    int32_t base;
-};
+// entries per direct-lookup quantizer table (one packed 32-bit word per bucket, see lt_api.cu)
 constexpr int kLutEntries = 4096;
 
 struct StepParams {
@@ -77,7 +73,7 @@ int ensure_device(cudaStream_t stream, DeviceInfo** out);
 // host copies of the code maps and of the search thresholds (mid-points rounded toward -inf)
 const float* host_table(bool is_signed);
 const float* host_mid_rd(bool is_signed);
-const QuantLut* host_lut(bool is_signed);   // nullptr if the maps do not fit the bucket grid
+const uint32_t* host_lut(bool is_signed);   // nullptr if the maps do not fit the bucket grid
 
 int launch_state_init(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
