@@ -164,12 +164,14 @@ static int validate_tensors(const lt_tensor* t, int32_t n, int need) {
 }
 
 // Packs tensors [*i, ...) into one launch's descriptors; advances *i.
-static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, StepParams* P, bool with_pg) {
+// param_dtype >= 0: only tensors whose parameters have that dtype (a launch is dtype-uniform).
+static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, StepParams* P, bool with_pg,
+                      int param_dtype) {
     int cnt = 0;
     int64_t blocks = 0;
     while (*i < n && cnt < kCap) {
         const lt_tensor& x = t[*i];
-        if (x.numel == 0) { ++*i; continue; }
+        if (x.numel == 0 || (param_dtype >= 0 && x.param_dtype != param_dtype)) { ++*i; continue; }
         const int64_t nb = (x.numel + block - 1) / block;
         if (blocks + nb > 0x7fffffff) break;   // next launch; one tensor alone always fits (numel <= 2^38)
         StepDesc& d = P->t[cnt];
@@ -236,10 +238,10 @@ int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt
     if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
     StepParams P;
     std::memset(&P.s, 0, sizeof(P.s));
-    P.sqnorm = nullptr; P.status = nullptr;
+    P.sqnorm = nullptr; P.status = nullptr; P.param_bf16 = 0;
     int32_t i = 0;
     while (i < n) {
-        pack_step(tensors, n, block, &i, &P, false);
+        pack_step(tensors, n, block, &i, &P, false, -1);
         if (P.n == 0) continue;
         if ((rc = launch_state_init(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
     }
@@ -322,11 +324,14 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
     P.s.precise_param = (hp->eps < 1e-15f) ? 1 : 0;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
-    int32_t i = 0;
-    while (i < n) {
-        pack_step(tensors, n, block, &i, &P, true);
-        if (P.n == 0) continue;
-        if ((rc = launch_step(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+    for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype per launch
+        P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
+        int32_t i = 0;
+        while (i < n) {
+            pack_step(tensors, n, block, &i, &P, true, dt);
+            if (P.n == 0) continue;
+            if ((rc = launch_step(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+        }
     }
     return LT_OK;
 }

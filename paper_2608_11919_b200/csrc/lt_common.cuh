@@ -44,6 +44,7 @@ struct StepParams {
     int32_t* status;
     int32_t n;
     int32_t total_blocks;
+    int32_t param_bf16;         // parameter dtype of every tensor of this launch
 };
 
 struct NormDesc {               // 24 bytes
