@@ -189,6 +189,8 @@ static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, 
             vec = vec && aligned(x.param, 4 * esize(x.param_dtype)) && aligned(x.grad, 4 * esize(x.grad_dtype));
         }
         if (vec) flags |= kFlagVecOk;
+        if (with_pg && aligned(x.param, 16) && aligned(x.grad, 16) && aligned(x.m_code, 16) && aligned(x.v_code, 16))
+            flags |= kFlagBulkOk;
         d.flags = flags;
         ++cnt; ++*i;
     }

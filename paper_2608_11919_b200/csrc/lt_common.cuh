@@ -15,6 +15,7 @@ constexpr int kCap = 480;
 constexpr int kFlagParamBf16 = 1;
 constexpr int kFlagGradF32 = 2;
 constexpr int kFlagVecOk = 4;   // every pointer allows 4-element vector access
+constexpr int kFlagBulkOk = 8;  // every pointer is 16-byte aligned (bulk prefetch of whole blocks allowed)
 
 struct StepDesc {               // 64 bytes
     void* p;
