@@ -108,6 +108,29 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 
+/* Largest number of non-empty tensors one lt_grad_sqnorm_multi_noalloc call accepts. */
+#define LT_NOALLOC_MAX_TENSORS 480
+
+/* (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * lt_grad_sqnorm_multi without a workspace argument. Some callers have no way to obtain device
+ * scratch at the point where they need the norm: code running under a framework allocator it must
+ * not call into, a region where cudaMalloc is forbidden because it would synchronise the device or
+ * break a capture in progress elsewhere in the process, or a plain C host that was handed gradient
+ * pointers and nothing else. For them the scratch (an arrival counter and up to 512 per-CTA partial
+ * sums, 4352 bytes) lives in a device array inside the library; every GPU that loads the library
+ * holds those bytes until the process exits. The call allocates and frees nothing, on host-visible
+ * CUDA APIs or otherwise.
+ *   - Same result contract as lt_grad_sqnorm_multi: ADDS the sum of squares to *d_sqnorm.
+ *   - At most LT_NOALLOC_MAX_TENSORS non-empty tensors per call (one launch over the fixed scratch);
+ *     more returns LT_ERR_WORKSPACE and enqueues nothing. Split longer lists over several calls.
+ *   - The first call on a device looks the array's device address up (and, if it is the library's
+ *     first call on that device at all, uploads the code tables and waits for that upload): make the
+ *     first call before any stream capture.
+ *   - All calls on a device share the one array. It keeps the previous call's contents; the call
+ *     clears the counter it needs at zero itself. Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on it and give wrong sums: order them. */
+int lt_grad_sqnorm_multi_noalloc(const lt_tensor* tensors, int32_t n, double* d_sqnorm, lt_stream stream);
+
 /* Name of a status code (static string). */
 const char* lt_status_str(int status);
 

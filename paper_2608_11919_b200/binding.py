@@ -50,6 +50,7 @@ def _load():
     L.lt_grad_sqnorm_multi.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
     L.lt_hybrid8_step.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_LtHParams), C.c_void_p,
                                   C.c_void_p, C.c_void_p]
+    L.lt_grad_sqnorm_multi_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     return L
 
 
@@ -153,6 +154,15 @@ def lt_grad_sqnorm_multi(tensors: TensorList, d_sqnorm: torch.Tensor, workspace:
     _check("lt_grad_sqnorm_multi",
            _lib.lt_grad_sqnorm_multi(tensors.ptr, tensors.n, d_sqnorm.data_ptr(), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def lt_grad_sqnorm_multi_noalloc(tensors: TensorList, d_sqnorm: torch.Tensor, stream=None) -> None:
+    """Squared-norm accumulation for callers that cannot provide device scratch: the library's own
+    fixed device array is used instead (shared by all calls on the device, so calls must not overlap
+    on the GPU; at most 480 non-empty tensors per call; first call before any stream capture)."""
+    assert d_sqnorm.dtype == torch.float64 and d_sqnorm.is_cuda
+    _check("lt_grad_sqnorm_multi_noalloc",
+           _lib.lt_grad_sqnorm_multi_noalloc(tensors.ptr, tensors.n, d_sqnorm.data_ptr(), _stream(stream)))
 
 
 def lt_hybrid8_step(tensors: TensorList, block: int, hp: HParams, d_sqnorm: Optional[torch.Tensor],

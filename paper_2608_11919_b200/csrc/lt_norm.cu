@@ -10,6 +10,8 @@
 // sum rounds. Per-CTA fp64 partials go to the workspace; the last CTA to arrive
 // (an atomic ticket, not a wait) adds them in index order and accumulates the launch total into
 // *out. Nothing depends on arrival order, so the result is bit-reproducible.
+#include <mutex>
+
 #include "lt_common.cuh"
 
 namespace lt {
@@ -143,3 +145,90 @@ int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s) {
 }
 
 }  // namespace lt
+
+// ---- lt_grad_sqnorm_multi_noalloc ------------------------------------------------------------------
+// Same kernel, scratch in a module-scope device array instead of a caller-supplied workspace.
+namespace {
+
+constexpr int kNoAllocMaxCtas = 512;                               // partial sums the array has room for
+constexpr int kNoAllocScratchBytes = 256 + kNoAllocMaxCtas * 8;    // arrival counter + partials: 4352 bytes
+
+// Every GPU that loads this library holds these 4352 bytes until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address, so the
+// address the kernel gets is asked for once per device (with that device current) and kept here.
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[64] = {nullptr};
+
+int noalloc_scratch(void** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LT_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (g_noalloc_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return LT_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return LT_OK;
+}
+
+}  // namespace
+
+extern "C" int lt_grad_sqnorm_multi_noalloc(const lt_tensor* tensors, int32_t n, double* d_sqnorm, lt_stream stream) {
+    using namespace lt;
+    if (n < 0 || (n > 0 && tensors == nullptr) || d_sqnorm == nullptr) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_sqnorm & 7) != 0) return LT_ERR_ALIGNMENT;
+    int live = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const lt_tensor& x = tensors[i];
+        if (x.numel < 0) return LT_ERR_INVALID_ARG;
+        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;
+        if (x.numel == 0) continue;
+        if ((x.grad_dtype != LT_F32 && x.grad_dtype != LT_BF16) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
+        if (((uintptr_t)x.grad % (x.grad_dtype == LT_F32 ? 4 : 2)) != 0) return LT_ERR_ALIGNMENT;
+        ++live;
+    }
+    if (live > LT_NOALLOC_MAX_TENSORS) return LT_ERR_WORKSPACE;   // beyond what one launch over the fixed scratch covers
+    if (live == 0) return LT_OK;
+
+    DeviceInfo* dev = nullptr;
+    int rc = ensure_device((cudaStream_t)stream, &dev);
+    if (rc != LT_OK) return rc;
+    void* scratch = nullptr;
+    if ((rc = noalloc_scratch(&scratch)) != LT_OK) return rc;
+
+    NormParams P;
+    P.ticket = (unsigned int*)scratch;
+    P.partials = (double*)((char*)scratch + 256);
+    P.out = d_sqnorm;
+    int cnt = 0;
+    int64_t items = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const lt_tensor& x = tensors[i];
+        if (x.numel == 0) continue;
+        const uintptr_t a = (uintptr_t)x.grad;
+        const int lead = (int)(a & 15);
+        const int64_t span = lead + x.numel * (x.grad_dtype == LT_F32 ? 4 : 2);
+        items += (span + kNormItemBytes - 1) / kNormItemBytes;
+        if (items > 0x7fffffff) return LT_ERR_UNSUPPORTED;
+        NormDesc& d = P.t[cnt++];
+        d.base16 = (const void*)(a - lead);
+        d.span_bytes = span;
+        d.item_end = (int32_t)items;
+        d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
+    }
+    P.n = cnt;
+    P.total_items = (int32_t)items;
+    // the array keeps what the last call left: the arrival counter must start at zero
+    if (cudaMemsetAsync(P.ticket, 0, 256, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
+    int grid = 2 * dev->sm_count;
+    if (grid > kNoAllocMaxCtas) grid = kNoAllocMaxCtas;
+    if (grid > P.total_items) grid = P.total_items;
+    sqnorm_kernel<<<grid, kNormThreads, 0, (cudaStream_t)stream>>>(P);
+    return cudaGetLastError() == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
