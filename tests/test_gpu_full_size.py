@@ -1,0 +1,116 @@
+"""Parity at the benchmark's full sizes (3B, 7B, 27B-shaped lists) in the launch configuration
+`bench.py` times: five GPU steps populate the state, then one more GPU step is compared against the
+oracle on sampled whole quantization blocks (every small tensor entirely; first, last and random
+blocks of every large tensor). The oracle's norm is its own fp64 sum over ALL gradients, streamed
+through the host. The full Ragged configuration (1000 tensors up to 4M elements, 10 free-running steps)
+is compared on a sampled subset of whole tensors the same way."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2608_11919_b200 as L
+from paper_2608_11919_b200 import workloads as W
+from parity_util import (NORM_RTOL, compare, oracle_sqnorm_of_buffers, oracle_tensors, parallel_oracle_step,
+                         refresh_grads)
+
+import bench
+
+pytestmark = pytest.mark.gpu
+WARM_STEPS = 5
+
+
+def sample_slices(spec, block, rng, per_tensor_blocks=24, small=1 << 16):
+    out = []
+    for t, size in enumerate(spec.sizes):
+        nb = (size + block - 1) // block
+        if size <= small:
+            out.append((t, 0, None))
+            continue
+        picks = {0, nb - 1} | set(int(x) for x in rng.integers(0, nb, per_tensor_blocks))
+        runs = sorted(picks)
+        out.append((t, runs[0], 2))                     # first two blocks
+        out.append((t, max(nb - 2, 0), 2))              # last two (the tail may be ragged)
+        for b in runs[1:-1]:
+            out.append((t, b, 1))
+    return out
+
+
+def run_full_size(name, block):
+    torch.cuda.set_device(0)
+    need = {"3b": 30e9, "7b": 70e9, "27b": 170e9}[name]
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip(f"{name}: needs {need / 1e9:.0f} GB of device memory, {free / 1e9:.0f} GB free")
+    spec, buf, opt = bench.build_workload(name, block, torch.device("cuda:0"))
+    for k in range(1, WARM_STEPS + 1):
+        W.fill_grads(buf, k)
+        opt.step()
+    torch.cuda.synchronize()
+    assert int(opt.status.item()) == 0
+    rng = np.random.default_rng(1234)
+    slices = sample_slices(spec, block, rng)
+    W.fill_grads(buf, WARM_STEPS + 1)
+    ots, slices = oracle_tensors(buf, slices=slices)     # state after the warm-up + this step's gradients
+    opt.step()
+    torch.cuda.synchronize()
+    S_gpu = float(opt.sqnorm.item())
+    S = oracle_sqnorm_of_buffers(buf)
+    assert abs(S_gpu - S) <= NORM_RTOL * S, (S_gpu, S)
+    ohp = O.HParams(max_norm=spec.max_norm, step=WARM_STEPS + 1)
+    assert parallel_oracle_step(ots, block, ohp, S) == 0
+    st = compare(buf, ots, slices)
+    st.norm_rel = abs(S_gpu - S) / S
+    print(name, block, "norm rel", st.norm_rel, st)
+    st.check()
+    assert st.n >= 2 * 10_000_000
+    del opt, buf
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("block", [2048, 4096])
+def test_3b_sampled_parity(block):
+    run_full_size("3b", block)
+
+
+def test_7b_sampled_parity():
+    run_full_size("7b", 2048)
+
+
+def test_27b_sampled_parity_chunked_bf16():
+    run_full_size("27b", 2048)
+
+
+def test_ragged_full_ten_steps_sampled_tensors():
+    torch.cuda.set_device(0)
+    block = 2048
+    spec = W.ragged_spec()                               # 1000 tensors, sizes up to 4M, seed 1
+    buf = W.Buffers(spec, block, "cuda:0")
+    W.fill_params(buf)
+    tl = L.TensorList.from_buffers(buf)
+    opt = L.Hybrid8Optimizer(tl, block, L.HParams(max_norm=spec.max_norm))
+    opt.init_state()
+    rng = np.random.default_rng(99)
+    order = rng.permutation(len(spec.sizes))
+    chosen, tot = [], 0
+    for t in order:                                      # whole tensors, about 12M elements in all
+        if tot + spec.sizes[t] <= 12_000_000:
+            chosen.append(int(t)); tot += spec.sizes[t]
+    chosen.sort()
+    W.fill_grads(buf, 1)
+    ots, slices = oracle_tensors(buf, indices=chosen)
+    ohp = O.HParams(max_norm=spec.max_norm)
+    for k in range(1, spec.steps + 1):
+        if k > 1:
+            W.fill_grads(buf, k)
+            refresh_grads(ots, buf, slices)
+        opt.step()
+        torch.cuda.synchronize()
+        S_gpu, S = float(opt.sqnorm.item()), oracle_sqnorm_of_buffers(buf)
+        assert abs(S_gpu - S) <= NORM_RTOL * S
+        ohp.step = k
+        parallel_oracle_step(ots, block, ohp, S)
+        st = compare(buf, ots, slices)
+        st.check()
+    print("ragged full:", spec.numel, "elements,", len(chosen), "tensors compared", st)
+    assert int(opt.status.item()) == 0
