@@ -14,8 +14,8 @@ namespace lt {
 struct HostTables {
     float qs[256], qu[256];
     float mid_s[256], mid_u[256];   // [k] = (T[k] + T[k+1]) / 2 rounded toward -inf; [255] = +inf
-    uint32_t lut_u[kLutEntries];    // see build_lut
-    uint32_t lut_s[kLutEntries];
+    uint32_t lut_u_full[lut_u_entries(true)], lut_s_full[lut_s_entries(true)];        // see build_lut
+    uint32_t lut_u_compact[lut_u_entries(false)], lut_s_compact[lut_s_entries(false)];
     bool lut_ok;
     HostTables() {
         static const double decade[7] = {1e-6, 1e-5, 1e-4, 1e-3, 1e-2, 1e-1, 1e0};
@@ -37,7 +37,8 @@ struct HostTables {
         qu[255] = 1.0f;
         fill_mid(qs, mid_s);
         fill_mid(qu, mid_u);
-        lut_ok = build_lut(mid_u, 7, false, lut_u) && build_lut(mid_s, 6, true, lut_s);
+        lut_ok = build_lut(mid_u, 7, false, 128, lut_u_full) && build_lut(mid_s, 6, true, 128, lut_s_full) &&
+                 build_lut(mid_u, 7, false, 32, lut_u_compact) && build_lut(mid_s, 6, true, 32, lut_s_compact);
     }
     static int code_of(const float* mid, float x) {   // number of thresholds strictly below x
         int c = 0;
@@ -45,25 +46,29 @@ struct HostTables {
         return c;
     }
     static float from_bits(uint32_t b) { float f; std::memcpy(&f, &b, 4); return f; }
-    // Direct-lookup form of the search. A bucket is the set of floats that share sign, exponent field
-    // (96..127, i.e. magnitude in [2^-31, 2)) and the top `mbits` mantissa bits; `frac` is the rest of
-    // the mantissa (fbits = 23 - mbits bits). The code map is so coarse against that grid that a
-    // bucket holds at most one threshold T, so code(x) = base + (x > T) with base = code of the
-    // bucket's smallest value. An entry packs both into one word so that ONE integer add decides:
-    //   x >= 0:  entry = base << 24 | (0xFFFFFF - frac(T));   code = (entry + frac(x)) >> 24
-    //            (the add carries into bits 24.. exactly when frac(x) > frac(T); no T: frac(T) = all ones)
-    //   x <  0:  entry = (base + 1) << 24 | frac(T);          code = (entry + ~frac(x)) >> 24
-    //            (= entry - frac(x) - 1, which keeps base + 1 exactly when frac(x) < frac(T), i.e. x > T;
-    //            no T: frac(T) = 0)
-    // Unsigned map: 32 x 128 buckets. Signed map: 32 x 64 buckets of the magnitude, positive half
-    // first, negative half second.
-    static bool build_lut(const float* mid, int mbits, bool is_signed, uint32_t* lut) {
-        const int per_binade = 1 << mbits, half = 32 * per_binade, fbits = 23 - mbits;
+    // Direct-lookup form of the search. A bucket is the set of floats below 2 that share sign,
+    // exponent field (0..127, subnormals included) and the top `mbits` mantissa bits; `frac` is the
+    // rest of the mantissa and H the bits above it (constant over the bucket). (A table may instead
+    // cover only exponent fields 96..127; the kernel then clamps smaller magnitudes up to 2^-31, which
+    // share the zero code.) The code map is so
+    // coarse against that grid that a bucket holds at most one threshold T, so code(x) = base +
+    // (x > T) with base = code of the bucket's smallest value. An entry packs both into one word so
+    // that ONE integer add of the magnitude bits a = |x| decides; the code is the top byte of the sum:
+    //   x >= 0:  entry = (base << 24 | 0xFFFFFF - frac(T)) - H;        sum = entry + a
+    //            (carries into bits 24.. exactly when frac(x) > frac(T); no T: frac(T) = all ones)
+    //   x <  0:  entry = ((base + 1) << 24 | frac(T)) + H;             sum = entry + ~a
+    //            (= (base + 1) << 24 + frac(T) - frac(x) - 1, which keeps base + 1 exactly when
+    //            frac(x) < frac(T), i.e. x > T; no T: frac(T) = 0)
+    // Unsigned map: 128 x 128 buckets. Signed map: 128 x 64 buckets of the magnitude, positive half
+    // first, negative half second. Exponent fields 128..255 (|x| >= 2, Inf, NaN) cannot occur for a
+    // normalised moment; the kernel masks the index so that even then the lookup stays inside the table.
+    static bool build_lut(const float* mid, int mbits, bool is_signed, int binades, uint32_t* lut) {
+        const int per_binade = 1 << mbits, half = binades * per_binade, fbits = 23 - mbits;
+        const int e_first = 128 - binades;   // first exponent field covered
         const uint32_t fmask = (1u << fbits) - 1u;
         for (int h = 0; h < (is_signed ? 2 : 1); ++h) {
             for (int key = 0; key < half; ++key) {
-                const uint32_t lo = ((uint32_t)(96 + key / per_binade) << 23) |
-                                    ((uint32_t)(key % per_binade) << fbits);
+                const uint32_t lo = ((uint32_t)(e_first + key / per_binade) << 23) | ((uint32_t)(key % per_binade) << fbits);
                 const uint32_t hi = lo | fmask;
                 const float xa = h == 0 ? from_bits(lo) : -from_bits(hi);   // smallest value of the bucket
                 const float xb = h == 0 ? from_bits(hi) : -from_bits(lo);   // largest
@@ -78,10 +83,10 @@ struct HostTables {
                 } else if (cb != ca) {
                     return false;
                 }
-                uint32_t e;
-                if (h == 0) e = ((uint32_t)ca << 24) | (0xFFFFFFu - (has_t ? tf : fmask));
-                else e = ((uint32_t)(ca + 1) << 24) | (has_t ? tf : 0u);
                 if (h == 1 && ca + 1 > 255) return false;
+                uint32_t e;
+                if (h == 0) e = (((uint32_t)ca << 24) | (0xFFFFFFu - (has_t ? tf : fmask))) - lo;
+                else e = (((uint32_t)(ca + 1) << 24) | (has_t ? tf : 0u)) + lo;
                 lut[h * half + key] = e;
             }
         }
@@ -105,9 +110,11 @@ static const HostTables& host_tables() {
 }
 const float* host_table(bool is_signed) { return is_signed ? host_tables().qs : host_tables().qu; }
 const float* host_mid_rd(bool is_signed) { return is_signed ? host_tables().mid_s : host_tables().mid_u; }
-const uint32_t* host_lut(bool is_signed) {
-    if (!host_tables().lut_ok) return nullptr;
-    return is_signed ? host_tables().lut_s : host_tables().lut_u;
+const uint32_t* host_lut(bool is_signed, bool full) {
+    const HostTables& t = host_tables();
+    if (!t.lut_ok) return nullptr;
+    if (full) return is_signed ? t.lut_s_full : t.lut_u_full;
+    return is_signed ? t.lut_s_compact : t.lut_u_compact;
 }
 
 // ---- per-device set-up ---------------------------------------------------------------------------

@@ -35,8 +35,13 @@ struct StepScalars {
     int32_t precise_param;      // 1: IEEE sqrt and divide in the parameter update (tiny eps)
 };
 
-// entries per direct-lookup quantizer table (one packed 32-bit word per bucket, see lt_api.cu)
-constexpr int kLutEntries = 4096;
+// Direct-lookup quantizer tables (one packed 32-bit word per bucket, see lt_api.cu). Two forms exist:
+// "full" covers every float below 2 (exponent fields 0..127: 128 binades, the input needs no clamping),
+// "compact" covers [2^-31, 2) (exponent fields 96..127: 32 binades, the kernel clamps smaller inputs up
+// to 2^-31, which share the zero code). The signed table has 64 buckets per binade and two halves
+// (positive, negative), the unsigned one 128 buckets per binade.
+constexpr int lut_s_entries(bool full) { return (full ? 128 : 32) * 64 * 2; }
+constexpr int lut_u_entries(bool full) { return (full ? 128 : 32) * 128; }
 
 struct StepParams {
     StepDesc t[kCap];
@@ -75,7 +80,7 @@ int ensure_device(cudaStream_t stream, DeviceInfo** out);
 // host copies of the code maps and of the search thresholds (mid-points rounded toward -inf)
 const float* host_table(bool is_signed);
 const float* host_mid_rd(bool is_signed);
-const uint32_t* host_lut(bool is_signed);   // nullptr if the maps do not fit the bucket grid
+const uint32_t* host_lut(bool is_signed, bool full);   // nullptr if the maps do not fit the bucket grid
 
 int launch_state_init(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
