@@ -29,9 +29,11 @@ if ROOT not in sys.path:
 
 METRIC = "optimizer-step params/s"
 UNIT = "params/s"
-# DRAM bytes per parameter of the fused step kernel measured with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum over one launch / parameters of that launch); see profiles/. None = not captured.
-STEP_TRAFFIC_BYTES_PER_PARAM = {"f32": None, "bf16": None}
+# DRAM bytes per parameter of the fused step kernel measured with ncu on the `small` workloads
+# (dram__bytes_read.sum + dram__bytes_write.sum of one launch / parameters of that launch, block 2048;
+# profiles/step_kernel_small.md). Traffic grows in proportion to the parameters, so a full launch's
+# traffic is this figure times its parameters.
+STEP_TRAFFIC_BYTES_PER_PARAM = {"f32": 14.10, "bf16": 9.93}
 
 
 def algorithmic_bytes_per_param(param_bytes: int, block: int):
@@ -298,6 +300,7 @@ def main():
     ap.add_argument("--block", type=int, default=2048)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-alt-block", action="store_true", help="skip the second run at the other block size")
     ap.add_argument("--cpu-sample", type=int, default=128 << 20, help="params in the oracle's timed sample")
     args = ap.parse_args()
 
@@ -353,6 +356,15 @@ def main():
             if i == 0:
                 raise
     h = results[head]
+    alt = None
+    if not dist_on and not args.no_alt_block:
+        alt_block = 4096 if args.block != 4096 else 2048      # the paper's block size beside the configs' one
+        try:
+            r2, _ = time_resident(head, alt_block, args.steps, args.warmup, rank, world, dist_on, sample_clocks=False)
+            alt = {"block": alt_block, "ms_per_step": r2["ms_per_step"], "params_per_s": r2["params_per_s"],
+                   "step_gbs": r2["step_gbs"], "whole_gbs": r2["whole_gbs"]}
+        except torch.OutOfMemoryError:
+            torch.cuda.empty_cache()
     e2e = None
     if not args.no_e2e:
         e2e = time_e2e(head, args.block, max(2, min(args.steps, 5)), args.warmup)
@@ -391,7 +403,7 @@ def main():
                            "parallelism": f"shard{world}+scalar-allreduce" if world > 1 else "single"},
                 "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": h["launches_per_step"] * args.steps, "clocks": h["clocks"],
-                "workloads": results, "notes": notes}
+                "other_block": alt, "workloads": results, "notes": notes}
         print(json.dumps(line))
     if dist_on:
         torch.distributed.destroy_process_group()

@@ -87,8 +87,14 @@ int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
 int upload_tables(cudaStream_t s);
 
-constexpr int kNormThreads = 512;
-constexpr int kNormVecPerThread = 4;
+#ifndef LT_NORM_THREADS
+#define LT_NORM_THREADS 512
+#define LT_NORM_VPT 4
+#define LT_NORM_CTAS 2
+#endif
+constexpr int kNormThreads = LT_NORM_THREADS;
+constexpr int kNormVecPerThread = LT_NORM_VPT;
+constexpr int kNormCtasPerSm = LT_NORM_CTAS;
 constexpr int kNormItemBytes = kNormThreads * kNormVecPerThread * 16;
 constexpr int kNormMaxCtas = 1024;
 constexpr int64_t kWorkspaceBytes = 256 + kNormMaxCtas * 8;

@@ -66,7 +66,7 @@ __device__ __forceinline__ double sq_partial(const char* base, int64_t off, int6
     return acc;
 }
 
-__global__ void __launch_bounds__(kNormThreads, 2) sqnorm_kernel(const __grid_constant__ NormParams P) {
+__global__ void __launch_bounds__(kNormThreads, kNormCtasPerSm) sqnorm_kernel(const __grid_constant__ NormParams P) {
     __shared__ double s_warp[kNormThreads / 32];
     __shared__ bool s_last;
     const int tid = threadIdx.x;
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kNormThreads, 2) sqnorm_kernel(const __grid_co
 }
 
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s) {
-    int grid = 2 * sm_count;
+    int grid = kNormCtasPerSm * sm_count;
     if (grid > kNormMaxCtas) grid = kNormMaxCtas;
     if (grid > p.total_items) grid = p.total_items;
     if (grid < 1) grid = 1;
@@ -226,7 +226,7 @@ extern "C" int lt_grad_sqnorm_multi_noalloc(const lt_tensor* tensors, int32_t n,
     P.total_items = (int32_t)items;
     // the array keeps what the last call left: the arrival counter must start at zero
     if (cudaMemsetAsync(P.ticket, 0, 256, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
-    int grid = 2 * dev->sm_count;
+    int grid = kNormCtasPerSm * dev->sm_count;
     if (grid > kNoAllocMaxCtas) grid = kNoAllocMaxCtas;
     if (grid > P.total_items) grid = P.total_items;
     sqnorm_kernel<<<grid, kNormThreads, 0, (cudaStream_t)stream>>>(P);
