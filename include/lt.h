@@ -41,6 +41,10 @@ typedef enum {
 
 typedef enum { LT_F32 = 0, LT_BF16 = 1 } lt_dtype;
 
+/* How a tensor's Adam moments are stored. The paper's measured configuration is a hybrid (Sec. 3.5 and the
+ * variant-configuration table): ordinary fp32 Adam states for most parameters, 8-bit states for a 2 % slice. */
+typedef enum { LT_STATE_U8 = 0, LT_STATE_F32 = 1 } lt_state_dtype;
+
 /* A CUDA stream handle (cudaStream_t / CUstream); NULL is the default stream. */
 typedef struct CUstream_st* lt_stream;
 
@@ -54,6 +58,10 @@ typedef struct {
     int64_t numel;        /* >= 0; a tensor with 0 elements is skipped                               */
     int32_t param_dtype;  /* lt_dtype                                                               */
     int32_t grad_dtype;   /* lt_dtype                                                               */
+    int32_t state_dtype;  /* lt_state_dtype. LT_STATE_F32: m_code and v_code point to float[numel]
+                             (4-byte aligned) holding the moments themselves; m_absmax / v_absmax are
+                             ignored and may be NULL; value-zero state is all zeros                    */
+    int32_t reserved;     /* set to 0                                                               */
 } lt_tensor;
 
 /* Hyper-parameters of one optimizer step (the paper's training-configuration table uses
@@ -101,6 +109,8 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  *     p  <- p (1 - lr wd) - lr / (1 - beta1^t) * m' / (sqrt(v') / sqrt(1 - beta2^t) + eps)
  *     per block: m_absmax = max |m'|, v_absmax = max v', codes = nearest map entry of m'/m_absmax,
  *     v'/v_absmax (ties to the lower index; an all-zero block gets zero codes and scale 0).
+ * Tensors with state_dtype LT_STATE_F32 get the same update with m, v read and written as fp32 (no
+ * tables, no block scales); both kinds may be mixed in one list and share the clip factor.
  * If S is NaN or Inf nothing is written except bit 0 of *d_status (the paper's "non-finite gradients
  * are skipped", training-configuration table); the caller clears d_status when it wants to.
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.

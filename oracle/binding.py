@@ -33,7 +33,8 @@ def build(force: bool = False) -> str:
 class _Tensor(C.Structure):
     _fields_ = [("param", C.c_void_p), ("grad", C.c_void_p), ("m_code", C.c_void_p), ("v_code", C.c_void_p),
                 ("m_absmax", C.c_void_p), ("v_absmax", C.c_void_p), ("numel", C.c_int64),
-                ("param_dtype", C.c_int32), ("grad_dtype", C.c_int32)]
+                ("param_dtype", C.c_int32), ("grad_dtype", C.c_int32), ("state_dtype", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class _HParams(C.Structure):
@@ -105,7 +106,7 @@ class OracleTensor:
     float32), m_code / v_code (uint8), m_absmax / v_absmax (float32, one per block)."""
 
     def __init__(self, param: np.ndarray, grad: np.ndarray, block: int,
-                 m_code=None, v_code=None, m_absmax=None, v_absmax=None):
+                 m_code=None, v_code=None, m_absmax=None, v_absmax=None, fp32_state: bool = False):
         self.param = np.ascontiguousarray(param).reshape(-1)
         self.grad = np.ascontiguousarray(grad).reshape(-1)
         assert self.param.dtype in (np.float32, np.uint16) and self.grad.dtype in (np.float32, np.uint16)
@@ -113,6 +114,13 @@ class OracleTensor:
         self.numel = int(self.param.size)
         self.block = int(block)
         nb = (self.numel + block - 1) // block
+        self.fp32_state = bool(fp32_state) or (m_code is not None and np.asarray(m_code).dtype == np.float32)
+        if self.fp32_state:       # plain fp32 moments live in m_code / v_code; the scale arrays are unused
+            self.m_code = np.zeros(self.numel, np.float32) if m_code is None else np.ascontiguousarray(m_code, np.float32)
+            self.v_code = np.zeros(self.numel, np.float32) if v_code is None else np.ascontiguousarray(v_code, np.float32)
+            self.m_absmax = np.zeros(nb, np.float32)
+            self.v_absmax = np.zeros(nb, np.float32)
+            return
         self.m_code = np.full(self.numel, 127, np.uint8) if m_code is None else np.ascontiguousarray(m_code, np.uint8)
         self.v_code = np.zeros(self.numel, np.uint8) if v_code is None else np.ascontiguousarray(v_code, np.uint8)
         self.m_absmax = np.zeros(nb, np.float32) if m_absmax is None else np.ascontiguousarray(m_absmax, np.float32)
@@ -136,7 +144,8 @@ class OracleTensor:
     def c(self) -> _Tensor:
         p = lambda a: a.ctypes.data_as(C.c_void_p)  # noqa: E731
         return _Tensor(p(self.param), p(self.grad), p(self.m_code), p(self.v_code), p(self.m_absmax),
-                       p(self.v_absmax), self.numel, self.param_dtype, self.grad_dtype)
+                       p(self.v_absmax), self.numel, self.param_dtype, self.grad_dtype,
+                       1 if self.fp32_state else 0, 0)
 
 
 def _carray(tensors):

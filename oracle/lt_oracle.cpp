@@ -130,6 +130,10 @@ struct lto_tensor {
     int64_t numel;
     int32_t param_dtype;  // 0 = fp32, 1 = bf16
     int32_t grad_dtype;
+    int32_t state_dtype;  // 0 = 8-bit codes + block scales; 1 = plain fp32 moments: m_code / v_code are
+                          //     float[numel] and the scale arrays are unused (the paper's "hybrid" split,
+                          //     Sec. 3.5: most parameters keep ordinary Adam states, a 2 % slice is 8-bit)
+    int32_t reserved;
 };
 
 struct lto_hparams {
@@ -206,6 +210,11 @@ void lto_step_scalars(const lto_hparams* hp, lto_scalars* s) {
 void lto_state_init(const lto_tensor* t, int32_t n, int32_t block) {
     for (int32_t k = 0; k < n; ++k) {
         const int64_t nb = (t[k].numel + block - 1) / block;
+        if (t[k].state_dtype == 1) {
+            float* m = (float*)t[k].m_code; float* v = (float*)t[k].v_code;
+            for (int64_t i = 0; i < t[k].numel; ++i) { m[i] = 0.0f; v[i] = 0.0f; }
+            continue;
+        }
         for (int64_t i = 0; i < t[k].numel; ++i) { t[k].m_code[i] = 127; t[k].v_code[i] = 0; }
         for (int64_t b = 0; b < nb; ++b) { t[k].m_absmax[b] = 0.0f; t[k].v_absmax[b] = 0.0f; }
     }
@@ -270,6 +279,33 @@ void lto_step_tensor(const lto_tensor* tt, int32_t block, const lto_scalars* s, 
     }
 }
 
+// O-7 applied to a tensor whose moments are plain fp32 arrays (state_dtype 1): the same element
+// arithmetic as O-5 without the table lines, and no O-6.
+void lto_step_tensor_fp32state(const lto_tensor* tt, const lto_scalars* s, float c) {
+    float* m = (float*)tt->m_code;
+    float* v = (float*)tt->v_code;
+    for (int64_t i = 0; i < tt->numel; ++i) {
+        const float g = load_elem(tt->grad, tt->grad_dtype, i) * c;
+        const float t1 = s->beta1 * m[i];
+        const float t2 = s->omb1 * g;
+        const float mm = t1 + t2;
+        const float gg = g * g;
+        const float t3 = s->beta2 * v[i];
+        const float t4 = s->omb2 * gg;
+        const float vv = t3 + t4;
+        const float sq = std::sqrt(vv);
+        const float t5 = sq * s->inv_sqrt_bc2;
+        const float den = t5 + s->eps;
+        const float q = mm / den;
+        const float p = load_elem(tt->param, tt->param_dtype, i);
+        const float t6 = p * s->decay;
+        const float t7 = s->step_size * q;
+        store_elem(tt->param, tt->param_dtype, i, t6 - t7);
+        m[i] = mm;
+        v[i] = vv;
+    }
+}
+
 // Whole step over a tensor list given the total squared norm S of ALL gradients of this optimizer
 // step (the list may be one chunk of them). Returns 0; *status bit 0 is set (and nothing else is
 // touched) when S is not finite.
@@ -280,7 +316,10 @@ int32_t lto_hybrid8_step(const lto_tensor* t, int32_t n, int32_t block, const lt
     if (nonfinite) { *status |= 1; return 0; }
     lto_scalars s;
     lto_step_scalars(hp, &s);
-    for (int32_t k = 0; k < n; ++k) lto_step_tensor(&t[k], block, &s, c, use_brute);
+    for (int32_t k = 0; k < n; ++k) {
+        if (t[k].state_dtype == 1) lto_step_tensor_fp32state(&t[k], &s, c);
+        else lto_step_tensor(&t[k], block, &s, c, use_brute);
+    }
     return 0;
 }
 

@@ -11,6 +11,7 @@ from typing import Optional, Sequence
 import torch
 
 LT_F32, LT_BF16 = 0, 1
+LT_STATE_U8, LT_STATE_F32 = 0, 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "liblt_hybrid8.so")
 
@@ -24,7 +25,8 @@ class LtError(RuntimeError):
 class _LtTensor(C.Structure):
     _fields_ = [("param", C.c_void_p), ("grad", C.c_void_p), ("m_code", C.c_void_p), ("v_code", C.c_void_p),
                 ("m_absmax", C.c_void_p), ("v_absmax", C.c_void_p), ("numel", C.c_int64),
-                ("param_dtype", C.c_int32), ("grad_dtype", C.c_int32)]
+                ("param_dtype", C.c_int32), ("grad_dtype", C.c_int32), ("state_dtype", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class _LtHParams(C.Structure):
@@ -102,9 +104,11 @@ class TensorList:
         for i in range(n):
             p, g = params[i], grads[i]
             assert p.is_contiguous() and g.is_contiguous() and p.numel() == g.numel()
+            st32 = m_codes[i].dtype == torch.float32        # plain fp32 moments instead of 8-bit codes
+            assert m_codes[i].dtype == v_codes[i].dtype and (st32 or m_codes[i].dtype == torch.uint8)
             self.array[i] = _LtTensor(p.data_ptr(), g.data_ptr(), m_codes[i].data_ptr(), v_codes[i].data_ptr(),
-                                      m_absmax[i].data_ptr(), v_absmax[i].data_ptr(), p.numel(),
-                                      _dt(p.dtype), _dt(g.dtype))
+                                      0 if st32 else m_absmax[i].data_ptr(), 0 if st32 else v_absmax[i].data_ptr(),
+                                      p.numel(), _dt(p.dtype), _dt(g.dtype), LT_STATE_F32 if st32 else LT_STATE_U8, 0)
 
     @classmethod
     def from_buffers(cls, buf, indices: Optional[Sequence[int]] = None) -> "TensorList":

@@ -1,0 +1,147 @@
+// The same clipped AdamW update for tensors whose moments are plain fp32 arrays (the larger part of
+// the paper's hybrid split, Sec. 3.5): read p, g, m, v, write p, m, v -- 26 bytes per parameter with
+// fp32 parameters and bf16 gradients, a pure HBM stream with no tables and no block exchange.
+//
+// Work item = 2048 consecutive elements of one tensor (items restart at every tensor); 256-thread CTAs
+// walk the items in a grid-stride loop, thread `tid` owning the 4-element groups (k * 256 + tid), k < 2,
+// so every warp-wide access is one contiguous run and all eight 16-byte loads of a thread are in flight
+// together. Moments are formed exactly as written (IEEE fp32, one rounding per operation, no fused
+// multiply-add), so the state matches a plain evaluation bit for bit; the parameter update uses the
+// approximate sqrt/reciprocal unless eps is tiny, as in the 8-bit kernel.
+#include <cuda_bf16.h>
+
+#include "lt_common.cuh"
+
+namespace lt {
+
+namespace {
+
+constexpr int kNT = 256;
+constexpr int kK = kAdamw32Item / (4 * kNT);
+
+struct Regs { float c, beta1, beta2, omb1, omb2, step_size, isb2, decay, eps; };
+
+__device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
+template <bool PRECISE>
+__device__ __forceinline__ float update(const Regs& r, float p, float g, float& m, float& v) {
+    const float gc = __fmul_rn(g, r.c);
+    m = __fadd_rn(__fmul_rn(r.beta1, m), __fmul_rn(r.omb1, gc));
+    v = __fadd_rn(__fmul_rn(r.beta2, v), __fmul_rn(r.omb2, __fmul_rn(gc, gc)));
+    if (PRECISE) {
+        const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), r.isb2), r.eps);
+        return __fsub_rn(__fmul_rn(p, r.decay), __fmul_rn(r.step_size, __fdiv_rn(m, den)));
+    }
+    const float den = __fmaf_rn(sqrt_approx(v), r.isb2, r.eps);
+    return __fmaf_rn(-r.step_size, __fmul_rn(m, rcp_approx(den)), __fmul_rn(p, r.decay));
+}
+
+template <bool PRECISE, bool P_BF16>
+__global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ StepParams P) {
+    const int tid = threadIdx.x;
+    Regs r;
+    r.c = 1.0f;
+    if (P.sqnorm != nullptr) {
+        const double S = *P.sqnorm;
+        if (!isfinite(S)) {
+            if (blockIdx.x == 0 && tid == 0 && P.status != nullptr) atomicOr(P.status, 1);
+            return;
+        }
+        if (P.s.clip_on) r.c = (float)fmin(1.0, (double)P.s.max_norm / (sqrt(S) + 1e-6));
+    }
+    r.beta1 = P.s.beta1; r.beta2 = P.s.beta2; r.omb1 = P.s.omb1; r.omb2 = P.s.omb2;
+    r.step_size = P.s.step_size; r.isb2 = P.s.inv_sqrt_bc2; r.decay = P.s.decay; r.eps = P.s.eps;
+
+    int t = 0, begin = 0;
+    for (int w = blockIdx.x; w < P.total_blocks; w += gridDim.x) {
+        while (w >= P.t[t].blk_end) { begin = P.t[t].blk_end; ++t; }
+        const StepDesc& d = P.t[t];
+        const int64_t e_base = (int64_t)(w - begin) * kAdamw32Item;
+        const int64_t rem = d.numel - e_base;
+        const int len = rem < kAdamw32Item ? (int)rem : kAdamw32Item;
+        const bool g_f32 = (d.flags & kFlagGradF32) != 0;
+        char* pp = (char*)d.p + e_base * (P_BF16 ? 2 : 4);
+        const char* gp = (const char*)d.g + e_base * (g_f32 ? 4 : 2);
+        float* mp = (float*)d.mc + e_base;
+        float* vp = (float*)d.vc + e_base;
+        if ((d.flags & kFlagVecOk) != 0 && !g_f32 && len == kAdamw32Item) {
+            uint4 pr[kK]; uint2 gr[kK]; float4 mr[kK], vr[kK];
+#pragma unroll
+            for (int k = 0; k < kK; ++k) {
+                const int e0 = (k * kNT + tid) * 4;
+                if (P_BF16) { const uint2 q = *(const uint2*)(pp + e0 * 2); pr[k].x = q.x; pr[k].y = q.y; }
+                else pr[k] = *(const uint4*)(pp + e0 * 4);
+                gr[k] = *(const uint2*)(gp + e0 * 2);
+                mr[k] = *(const float4*)(mp + e0);
+                vr[k] = *(const float4*)(vp + e0);
+            }
+#pragma unroll
+            for (int k = 0; k < kK; ++k) {
+                const int e0 = (k * kNT + tid) * 4;
+                float p[4], g[4], pn[4];
+                if (P_BF16) {
+                    p[0] = __uint_as_float(pr[k].x << 16); p[1] = __uint_as_float(pr[k].x & 0xffff0000u);
+                    p[2] = __uint_as_float(pr[k].y << 16); p[3] = __uint_as_float(pr[k].y & 0xffff0000u);
+                } else {
+                    p[0] = __uint_as_float(pr[k].x); p[1] = __uint_as_float(pr[k].y);
+                    p[2] = __uint_as_float(pr[k].z); p[3] = __uint_as_float(pr[k].w);
+                }
+                g[0] = __uint_as_float(gr[k].x << 16); g[1] = __uint_as_float(gr[k].x & 0xffff0000u);
+                g[2] = __uint_as_float(gr[k].y << 16); g[3] = __uint_as_float(gr[k].y & 0xffff0000u);
+                pn[0] = update<PRECISE>(r, p[0], g[0], mr[k].x, vr[k].x);
+                pn[1] = update<PRECISE>(r, p[1], g[1], mr[k].y, vr[k].y);
+                pn[2] = update<PRECISE>(r, p[2], g[2], mr[k].z, vr[k].z);
+                pn[3] = update<PRECISE>(r, p[3], g[3], mr[k].w, vr[k].w);
+                if (P_BF16) {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(pn[0], pn[1]);
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(pn[2], pn[3]);
+                    uint2 q;
+                    q.x = *reinterpret_cast<const uint32_t*>(&lo);
+                    q.y = *reinterpret_cast<const uint32_t*>(&hi);
+                    *(uint2*)(pp + e0 * 2) = q;
+                } else {
+                    *(float4*)(pp + e0 * 4) = make_float4(pn[0], pn[1], pn[2], pn[3]);
+                }
+                *(float4*)(mp + e0) = mr[k];
+                *(float4*)(vp + e0) = vr[k];
+            }
+        } else {
+            for (int e = tid; e < len; e += kNT) {
+                const float p = P_BF16 ? __uint_as_float((uint32_t)*(const unsigned short*)(pp + e * 2) << 16)
+                                       : *(const float*)(pp + e * 4);
+                const float g = g_f32 ? *(const float*)(gp + e * 4)
+                                      : __uint_as_float((uint32_t)*(const unsigned short*)(gp + e * 2) << 16);
+                float m = mp[e], v = vp[e];
+                const float pn = update<PRECISE>(r, p, g, m, v);
+                if (P_BF16) *(unsigned short*)(pp + e * 2) = __bfloat16_as_ushort(__float2bfloat16_rn(pn));
+                else *(float*)(pp + e * 4) = pn;
+                mp[e] = m;
+                vp[e] = v;
+            }
+        }
+    }
+}
+
+template <bool PRECISE, bool P_BF16>
+int launch(const StepParams& p, int sm_count, cudaStream_t s) {
+    static int full_grid = 0;
+    if (full_grid == 0) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adamw32_kernel<PRECISE, P_BF16>, kNT, 0) != cudaSuccess ||
+            per_sm < 1) { cudaGetLastError(); return LT_ERR_CUDA; }
+        full_grid = per_sm * sm_count;
+    }
+    const int grid = p.total_blocks < full_grid ? p.total_blocks : full_grid;
+    adamw32_kernel<PRECISE, P_BF16><<<grid, kNT, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s) {
+    if (p.param_bf16) return p.s.precise_param ? launch<true, true>(p, sm_count, s) : launch<false, true>(p, sm_count, s);
+    return p.s.precise_param ? launch<true, false>(p, sm_count, s) : launch<false, false>(p, sm_count, s);
+}
+
+}  // namespace lt

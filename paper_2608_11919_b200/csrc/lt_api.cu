@@ -163,8 +163,14 @@ static int validate_tensors(const lt_tensor* t, int32_t n, int need) {
             if (!aligned(x.param, esize(x.param_dtype))) return LT_ERR_ALIGNMENT;
         }
         if (need & NEED_STATE) {
-            if (!x.m_code || !x.v_code || !x.m_absmax || !x.v_absmax) return LT_ERR_INVALID_ARG;
-            if (!aligned(x.m_absmax, 4) || !aligned(x.v_absmax, 4)) return LT_ERR_ALIGNMENT;
+            if (x.state_dtype != LT_STATE_U8 && x.state_dtype != LT_STATE_F32) return LT_ERR_INVALID_ARG;
+            if (!x.m_code || !x.v_code) return LT_ERR_INVALID_ARG;
+            if (x.state_dtype == LT_STATE_F32) {
+                if (!aligned(x.m_code, 4) || !aligned(x.v_code, 4)) return LT_ERR_ALIGNMENT;
+            } else {
+                if (!x.m_absmax || !x.v_absmax) return LT_ERR_INVALID_ARG;
+                if (!aligned(x.m_absmax, 4) || !aligned(x.v_absmax, 4)) return LT_ERR_ALIGNMENT;
+            }
         }
     }
     return LT_OK;
@@ -172,13 +178,15 @@ static int validate_tensors(const lt_tensor* t, int32_t n, int need) {
 
 // Packs tensors [*i, ...) into one launch's descriptors; advances *i.
 // param_dtype >= 0: only tensors whose parameters have that dtype (a launch is dtype-uniform).
+// state_dtype >= 0: only tensors with that kind of moments.
 static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, StepParams* P, bool with_pg,
-                      int param_dtype) {
+                      int param_dtype, int state_dtype = -1) {
     int cnt = 0;
     int64_t blocks = 0;
     while (*i < n && cnt < kCap) {
         const lt_tensor& x = t[*i];
-        if (x.numel == 0 || (param_dtype >= 0 && x.param_dtype != param_dtype)) { ++*i; continue; }
+        if (x.numel == 0 || (param_dtype >= 0 && x.param_dtype != param_dtype) ||
+            (state_dtype >= 0 && x.state_dtype != state_dtype)) { ++*i; continue; }
         const int64_t nb = (x.numel + block - 1) / block;
         if (blocks + nb > 0x7fffffff) break;   // next launch; one tensor alone always fits (numel <= 2^38)
         StepDesc& d = P->t[cnt];
@@ -189,7 +197,9 @@ static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, 
         blocks += nb;
         d.blk_end = (int32_t)blocks;
         int flags = 0;
-        bool vec = aligned(x.m_code, 4) && aligned(x.v_code, 4);
+        const bool st32 = x.state_dtype == LT_STATE_F32;
+        if (st32) flags |= kFlagStateF32;
+        bool vec = st32 ? (aligned(x.m_code, 16) && aligned(x.v_code, 16)) : (aligned(x.m_code, 4) && aligned(x.v_code, 4));
         if (with_pg) {
             if (x.param_dtype == LT_BF16) flags |= kFlagParamBf16;
             if (x.grad_dtype == LT_F32) flags |= kFlagGradF32;
@@ -333,13 +343,17 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
     P.s.precise_param = (hp->eps < 1e-15f) ? 1 : 0;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
-    for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype per launch
-        P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
-        int32_t i = 0;
-        while (i < n) {
-            pack_step(tensors, n, block, &i, &P, true, dt);
-            if (P.n == 0) continue;
-            if ((rc = launch_step(P, block, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
+    for (int st = LT_STATE_U8; st <= LT_STATE_F32; ++st) {
+        for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype and one state kind per launch
+            P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
+            int32_t i = 0;
+            while (i < n) {
+                pack_step(tensors, n, st == LT_STATE_F32 ? kAdamw32Item : block, &i, &P, true, dt, st);
+                if (P.n == 0) continue;
+                rc = st == LT_STATE_F32 ? launch_adamw32(P, dev->sm_count, (cudaStream_t)stream)
+                                        : launch_step(P, block, dev->sm_count, (cudaStream_t)stream);
+                if (rc != LT_OK) return rc;
+            }
         }
     }
     return LT_OK;

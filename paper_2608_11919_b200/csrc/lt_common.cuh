@@ -15,6 +15,7 @@ constexpr int kCap = 480;
 constexpr int kFlagParamBf16 = 1;
 constexpr int kFlagGradF32 = 2;
 constexpr int kFlagVecOk = 4;   // every pointer allows 4-element vector access
+constexpr int kFlagStateF32 = 16; // moments are plain fp32 arrays (mc / vc point to float)
 constexpr int kFlagBulkOk = 8;  // every pointer is 16-byte aligned (bulk prefetch of whole blocks allowed)
 
 struct StepDesc {               // 64 bytes
@@ -84,6 +85,8 @@ const uint32_t* host_lut(bool is_signed, bool full);   // nullptr if the maps do
 
 int launch_state_init(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
+int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s);   // tensors with fp32 moments
+constexpr int kAdamw32Item = 2048;   // elements per work item of that kernel (items restart at every tensor)
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
 int upload_tables(cudaStream_t s);
 

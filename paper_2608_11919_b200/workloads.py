@@ -51,6 +51,7 @@ class Spec:
     steps: int = 3
     step_scale: dict = field(default_factory=dict)   # {step: factor} applied to that step's grads
     align_elems: int = 1             # each tensor's offset in the flat buffers is a multiple of this
+    state_f32: Optional[List[bool]] = None   # per tensor: plain fp32 moments instead of 8-bit codes (hybrid split)
 
     @property
     def numel(self) -> int:
@@ -143,7 +144,8 @@ def small_bf16_spec() -> Spec:
     return s
 
 
-SPECS = {"small": small_spec, "small_bf16": small_bf16_spec, "tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
+SPECS = {"7b_hybrid": lambda: hybrid_split(qwen7b_spec()), "small_hybrid": lambda: hybrid_split(small_spec()),
+         "small": small_spec, "small_bf16": small_bf16_spec, "tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
 
 
 def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:
@@ -157,38 +159,74 @@ def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:
 
 class Buffers:
     """Flat device (or host) buffers for one workload; tensor t occupies [off[t], off[t]+size[t]) of
-    param / grad / m_code / v_code and [boff[t], boff[t]+nb[t]) of the two scale arrays."""
+    param / grad. Tensors with 8-bit state own [off8[t], ...) of m_code / v_code and [boff[t], boff[t]+nb[t])
+    of the two scale arrays; tensors with fp32 state own [off32[t], ...) of m_f32 / v_f32."""
 
     def __init__(self, spec: Spec, block: int, device, pin: bool = False):
         self.spec, self.block, self.device = spec, int(block), torch.device(device)
         a = spec.align_elems
-        self.off, self.boff = [], []
-        o = b = 0
-        for s in spec.sizes:
+        self.f32 = list(spec.state_f32) if spec.state_f32 is not None else [False] * len(spec.sizes)
+        self.off, self.boff, self.off8, self.off32 = [], [], [], []
+        o = b = o8 = o32 = 0
+        for s, f in zip(spec.sizes, self.f32):
             o = (o + a - 1) // a * a
-            self.off.append(o); self.boff.append(b)
-            o += s; b += (s + block - 1) // block
+            o8 = (o8 + a - 1) // a * a
+            o32 = (o32 + a - 1) // a * a
+            self.off.append(o); self.boff.append(b); self.off8.append(o8); self.off32.append(o32)
+            o += s
+            if f:
+                o32 += s
+            else:
+                o8 += s; b += (s + block - 1) // block
         self.total, self.total_blocks = o, b
         kw = dict(device=self.device)
         if pin and self.device.type == "cpu":
             kw["pin_memory"] = True
         self.param = torch.empty(max(o, 1), dtype=spec.param_dtype, **kw)
         self.grad = torch.empty(max(o, 1), dtype=spec.grad_dtype, **kw)
-        self.m_code = torch.empty(max(o, 1), dtype=torch.uint8, **kw)
-        self.v_code = torch.empty(max(o, 1), dtype=torch.uint8, **kw)
+        self.m_code = torch.empty(max(o8, 1), dtype=torch.uint8, **kw)
+        self.v_code = torch.empty(max(o8, 1), dtype=torch.uint8, **kw)
         self.m_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
         self.v_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
+        self.m_f32 = torch.empty(max(o32, 1), dtype=torch.float32, **kw)
+        self.v_f32 = torch.empty(max(o32, 1), dtype=torch.float32, **kw)
 
     def view(self, which: str, t: int) -> torch.Tensor:
-        buf = getattr(self, which)
+        size = self.spec.sizes[t]
         if which in ("m_absmax", "v_absmax"):
-            nb = (self.spec.sizes[t] + self.block - 1) // self.block
-            return buf[self.boff[t]: self.boff[t] + nb]
-        return buf[self.off[t]: self.off[t] + self.spec.sizes[t]]
+            nb = 0 if self.f32[t] else (size + self.block - 1) // self.block
+            return getattr(self, which)[self.boff[t]: self.boff[t] + nb]
+        if which in ("m_code", "v_code"):          # the moment storage, whichever kind this tensor has
+            if self.f32[t]:
+                return (self.m_f32 if which == "m_code" else self.v_f32)[self.off32[t]: self.off32[t] + size]
+            return getattr(self, which)[self.off8[t]: self.off8[t] + size]
+        return getattr(self, which)[self.off[t]: self.off[t] + size]
 
     def resident_bytes(self) -> int:
         return sum(getattr(self, k).numel() * getattr(self, k).element_size()
-                   for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax"))
+                   for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax", "m_f32", "v_f32"))
+
+
+def hybrid_split(spec: Spec, eight_bit_fraction: float = 0.02) -> Spec:
+    """Marks tensors as fp32-state so that about `eight_bit_fraction` of the parameters keep 8-bit state
+    (the paper's hybrid configuration: a 2 % 8-bit slice, ordinary Adam states elsewhere). The 8-bit slice
+    is taken from the smaller matrices of the last layers until the fraction is reached."""
+    target = eight_bit_fraction * spec.numel
+    order = sorted(range(len(spec.sizes)), key=lambda i: (-spec.layer_of[i], spec.sizes[i]))
+    f32 = [True] * len(spec.sizes)
+    got = 0
+    for i in order:
+        if spec.layer_of[i] < 0 or spec.sizes[i] < 4096:
+            continue
+        if got + spec.sizes[i] > 1.25 * target:
+            continue
+        f32[i] = False
+        got += spec.sizes[i]
+        if got >= target:
+            break
+    spec.state_f32 = f32
+    spec.name = spec.name + "_hybrid"
+    return spec
 
 
 def _gen(device, seed: int) -> torch.Generator:

@@ -42,7 +42,8 @@ def oracle_tensors(buf: W.Buffers, indices=None, slices=None):
         out.append(O.OracleTensor(
             host_np(buf.view("param", t)[e0:e1]), host_np(buf.view("grad", t)[e0:e1]), buf.block,
             host_np(buf.view("m_code", t)[e0:e1]), host_np(buf.view("v_code", t)[e0:e1]),
-            host_np(buf.view("m_absmax", t)[b0:b1]), host_np(buf.view("v_absmax", t)[b0:b1])))
+            None if buf.f32[t] else host_np(buf.view("m_absmax", t)[b0:b1]),
+            None if buf.f32[t] else host_np(buf.view("v_absmax", t)[b0:b1])))
     return out, slices
 
 
@@ -74,6 +75,7 @@ class Stats:
         self.scale_max_rel = 0.0
         self.code_mismatch = 0
         self.code_max_dist = 0
+        self.state32_max_rel = 0.0      # fp32 moments of tensors with plain fp32 state
 
     def __repr__(self):
         return (f"Stats(n={self.n}, param_max_rel={self.param_max_rel:.3g}, param_max_ulp={self.param_max_ulp}, "
@@ -84,6 +86,7 @@ class Stats:
         assert self.param_max_rel <= PARAM_RTOL, self
         assert self.param_max_ulp <= 1, self
         assert self.scale_max_rel <= SCALE_RTOL, self
+        assert self.state32_max_rel <= SCALE_RTOL, self
         assert self.code_max_dist <= 1, self
         assert self.code_mismatch <= (1.0 - CODE_MATCH_MIN) * max(self.n, 1), self
 
@@ -108,6 +111,15 @@ def compare(buf: W.Buffers, ots, slices, stats: Stats | None = None) -> Stats:
         else:
             if n:
                 st.param_max_ulp = max(st.param_max_ulp, int(np.abs(_bf16_ordinal(gp) - _bf16_ordinal(ot.param)).max()))
+        if ot.fp32_state:                 # plain fp32 moments: compared as values
+            for key in ("m_code", "v_code"):
+                g = host_np(buf.view(key, t)[e0:e0 + n]).astype(np.float64)
+                r = getattr(ot, key).astype(np.float64)
+                if n:
+                    rel = np.abs(g - r) / np.maximum(np.abs(r), 1e-30)
+                    st.state32_max_rel = max(st.state32_max_rel, float(np.where(g == r, 0.0, rel).max()))
+            st.n += 2 * n
+            continue
         for key in ("m_absmax", "v_absmax"):
             g = host_np(buf.view(key, t)[b0:b0 + nbk]).astype(np.float64)
             r = getattr(ot, key).astype(np.float64)

@@ -39,7 +39,7 @@ def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True)
     W.fill_grads(buf, 1)
     ots, slices = oracle_tensors(buf)
     # S0 parity: the kernel's initial state equals the oracle's
-    init = [O.OracleTensor(t.param.copy(), t.grad.copy(), block) for t in ots]
+    init = [O.OracleTensor(t.param.copy(), t.grad.copy(), block, fp32_state=t.fp32_state) for t in ots]
     O.state_init(init, block)
     for a, b in zip(ots, init):
         for k in ("m_code", "v_code", "m_absmax", "v_absmax"):
@@ -258,3 +258,20 @@ def test_resume_from_saved_state_is_bit_identical():
     torch.cuda.synchronize()
     for key in ("m_code", "v_code", "m_absmax", "v_absmax", "param"):
         assert torch.equal(getattr(a, key), getattr(b, key)), key
+
+
+def test_hybrid_fp32_and_8bit_state_in_one_list():
+    # the paper's hybrid split: most tensors keep plain fp32 moments, a slice is 8-bit; one call updates both
+    for pd in (torch.float32, torch.bfloat16):
+        spec = W.ragged_spec(n_tensors=120, max_numel=1 << 16, seed=13)
+        spec.param_dtype = pd
+        spec.state_f32 = [i % 3 != 0 for i in range(len(spec.sizes))]
+        stats = run_free(spec, 4096, 4)
+        assert stats[-1].state32_max_rel == 0.0          # fp32 moments are bit-identical
+
+
+def test_hybrid_decoder_split_matches_target_fraction():
+    spec = W.hybrid_split(W.small_spec())
+    n8 = sum(s for s, f in zip(spec.sizes, spec.state_f32) if not f)
+    assert 0.015 <= n8 / spec.numel <= 0.03
+    run_free(spec, 4096, 2, check_every_step=False)

@@ -506,3 +506,37 @@ def test_quantized_trajectory_stays_near_fp32_trajectory():
         assert np.max(np.abs(vq - v)) <= 0.03 * k * np.max(v)
         # every parameter moved by at most ~lr per step in both, so they stay within 2*k*lr
         assert np.max(np.abs(t.param - p)) <= 2 * k * 1e-5
+
+
+# ---------------------------------------------------------------------------------------------
+# hybrid split: tensors with plain fp32 moments inside the same step
+# ---------------------------------------------------------------------------------------------
+def test_fp32_state_tensors_in_the_step_equal_the_pinned_fp32_mode():
+    rng = np.random.default_rng(21)
+    n = 3000
+    p0 = rng.normal(0, 0.02, n).astype(np.float32)
+    t32 = O.OracleTensor(p0.copy(), np.zeros(n, np.uint16), 4096, fp32_state=True)
+    t8 = O.OracleTensor(p0.copy(), np.zeros(n, np.uint16), 4096)
+    tb = O.OracleTensor(O.f32_to_bf16_bits(p0), np.zeros(n, np.uint16), 4096, fp32_state=True)
+    p = p0.copy(); m = np.zeros(n, np.float32); v = np.zeros(n, np.float32)
+    pb = bf16_round(p0); mb = np.zeros(n, np.float32); vb = np.zeros(n, np.float32)
+    hp = paper_hp(max_norm=0.5)
+    for k in (1, 2, 3):
+        g = O.f32_to_bf16_bits(rng.normal(0, 1e-3, n).astype(np.float32))
+        for t in (t32, t8, tb):
+            t.set_grad(g)
+        S = O.sqnorm([t32, t8])
+        c, _ = O.clip_factor(S, hp.max_norm)
+        hp.step = k
+        assert O.hybrid8_step([t32, t8, tb], 4096, hp, S) == 0       # mixed list, one clip factor
+        O.step_fp32state(p, O.bf16_bits_to_f32(g), m, v, hp, c)      # the mode pinned against torch.optim.AdamW
+        assert np.array_equal(t32.param, p) and np.array_equal(t32.m_code, m) and np.array_equal(t32.v_code, v)
+        # bf16 parameters: same moments, parameter = RNE of the fp32 result computed from the bf16 parameter
+        O.step_fp32state(pb, O.bf16_bits_to_f32(g), mb, vb, hp, c)
+        assert np.array_equal(tb.param, O.f32_to_bf16_bits(pb))
+        pb = bf16_round(pb)
+        assert np.array_equal(tb.m_code, m)
+    assert t8.m_code.dtype == np.uint8 and not np.array_equal(t8.param, p0)
+    z = O.OracleTensor(p0.copy(), np.zeros(n, np.uint16), 4096, m_code=np.ones(n, np.float32), v_code=np.ones(n, np.float32))
+    O.state_init([z], 4096)
+    assert not z.m_code.any() and not z.v_code.any()
