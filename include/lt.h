@@ -118,6 +118,21 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 
+/* Per-tensor squared L2 norms, for logging (Sec. 3.5: the clip "computes per-tensor norms" before it
+ * aggregates them). ADDS sum_i grad[t][i]^2 to d_out[t] for every tensor t of the list (device doubles,
+ * one per list entry, zeroed by the caller; entries of empty tensors are left alone). Uses grad,
+ * grad_dtype, numel. Each addend is an exact fp64 square; per-CTA partial sums reach d_out[t] through
+ * fp64 atomic adds, so the last bits may differ from run to run -- use lt_grad_sqnorm_multi for the norm
+ * that feeds the clip. No workspace. */
+int lt_grad_sqnorm_per_tensor(const lt_tensor* tensors, int32_t n, double* d_out, lt_stream stream);
+
+/* Skip bookkeeping, once per optimizer step, after the step's norm is complete (training-configuration
+ * table: "Non-finite gradients are skipped; training aborts after three consecutive non-finite-gradient
+ * events"). Reads S = *d_sqnorm and updates the device word *d_skip_count: S finite -> 0, S NaN/Inf ->
+ * previous value + 1. The caller reads it when it likes and applies its abort policy; nothing here
+ * aborts. One thread of device work. */
+int lt_skip_count_update(const double* d_sqnorm, int32_t* d_skip_count, lt_stream stream);
+
 /* Largest number of non-empty tensors one lt_grad_sqnorm_multi_noalloc call accepts. */
 #define LT_NOALLOC_MAX_TENSORS 480
 

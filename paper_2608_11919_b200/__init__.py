@@ -9,7 +9,7 @@ of any entry point loads the library and raises ImportError if it has not been b
 _BINDING_NAMES = (
     "LT_F32", "LT_BF16", "LtError", "HParams", "TensorList", "library_path",
     "lt_hybrid8_state_bytes", "lt_hybrid8_code_table", "lt_workspace_bytes", "lt_hybrid8_state_init",
-    "lt_grad_sqnorm_multi", "lt_grad_sqnorm_multi_noalloc", "lt_hybrid8_step", "lt_status_str",
+    "lt_grad_sqnorm_multi", "lt_grad_sqnorm_multi_noalloc", "lt_grad_sqnorm_per_tensor", "lt_skip_count_update", "lt_hybrid8_step", "lt_status_str",
     "Hybrid8Optimizer",
 )
 __all__ = list(_BINDING_NAMES)

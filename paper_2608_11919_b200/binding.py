@@ -53,6 +53,8 @@ def _load():
     L.lt_hybrid8_step.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_LtHParams), C.c_void_p,
                                   C.c_void_p, C.c_void_p]
     L.lt_grad_sqnorm_multi_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    L.lt_grad_sqnorm_per_tensor.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    L.lt_skip_count_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     return L
 
 
@@ -169,6 +171,18 @@ def lt_grad_sqnorm_multi_noalloc(tensors: TensorList, d_sqnorm: torch.Tensor, st
            _lib.lt_grad_sqnorm_multi_noalloc(tensors.ptr, tensors.n, d_sqnorm.data_ptr(), _stream(stream)))
 
 
+def lt_grad_sqnorm_per_tensor(tensors: TensorList, d_out: torch.Tensor, stream=None) -> None:
+    assert d_out.dtype == torch.float64 and d_out.is_cuda and d_out.numel() >= tensors.n
+    _check("lt_grad_sqnorm_per_tensor",
+           _lib.lt_grad_sqnorm_per_tensor(tensors.ptr, tensors.n, d_out.data_ptr(), _stream(stream)))
+
+
+def lt_skip_count_update(d_sqnorm: torch.Tensor, d_skip_count: torch.Tensor, stream=None) -> None:
+    assert d_sqnorm.dtype == torch.float64 and d_skip_count.dtype == torch.int32
+    _check("lt_skip_count_update",
+           _lib.lt_skip_count_update(d_sqnorm.data_ptr(), d_skip_count.data_ptr(), _stream(stream)))
+
+
 def lt_hybrid8_step(tensors: TensorList, block: int, hp: HParams, d_sqnorm: Optional[torch.Tensor],
                     d_status: Optional[torch.Tensor], stream=None) -> None:
     h = hp.c()
@@ -190,6 +204,7 @@ class Hybrid8Optimizer:
         self.sqnorm = torch.zeros(1, dtype=torch.float64, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.workspace = torch.empty(lt_workspace_bytes(), dtype=torch.uint8, device=device)
+        self.skip_count = torch.zeros(1, dtype=torch.int32, device=device)   # consecutive non-finite steps
         self.t = 0
 
     def init_state(self) -> None:
@@ -201,5 +216,6 @@ class Hybrid8Optimizer:
         self.sqnorm.zero_()
         for ch in self.chunks:
             lt_grad_sqnorm_multi(ch, self.sqnorm, self.workspace)
+        lt_skip_count_update(self.sqnorm, self.skip_count)
         for ch in self.chunks:
             lt_hybrid8_step(ch, self.block, self.hp, self.sqnorm, self.status)

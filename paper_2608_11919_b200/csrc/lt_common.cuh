@@ -54,11 +54,13 @@ struct StepParams {
     int32_t param_bf16;         // parameter dtype of every tensor of this launch
 };
 
-struct NormDesc {               // 24 bytes
+struct NormDesc {               // 32 bytes
     const void* base16;         // gradient address rounded down to 16 bytes
     int64_t span_bytes;         // lead bytes + numel * element size
     int32_t item_end;           // exclusive end of this tensor's range of launch-wide work items
     int32_t lead_f32;           // lead bytes (0..15) | grad_is_f32 << 8
+    int32_t slot;               // per-tensor output index (per-tensor norm kernel only)
+    int32_t pad;
 };
 
 struct NormParams {

@@ -146,6 +146,115 @@ int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s) {
 
 }  // namespace lt
 
+// ---- per-tensor norms and skip bookkeeping -----------------------------------------------------------
+namespace lt {
+
+// Same item walk as sqnorm_kernel; a CTA flushes its running sum to the tensor's slot whenever the item
+// it picks up belongs to another tensor (and at the end), so atomics are few.
+__global__ void __launch_bounds__(kNormThreads, 2) sqnorm_per_tensor_kernel(const __grid_constant__ NormParams P) {
+    __shared__ double s_warp[kNormThreads / 32];
+    const int tid = threadIdx.x;
+    double acc = 0.0;
+    int t = 0, item_begin = 0, cur = -1;
+    for (int w = blockIdx.x; ; w += gridDim.x) {
+        const bool more = w < P.total_items;
+        if (more) while (w >= P.t[t].item_end) { item_begin = P.t[t].item_end; ++t; }
+        if (cur >= 0 && (!more || t != cur)) {      // flush the finished tensor's partial sum
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            __syncthreads();
+            if ((tid & 31) == 0) s_warp[tid >> 5] = acc;
+            __syncthreads();
+            if (tid == 0) {
+                double s = 0.0;
+                for (int i = 0; i < kNormThreads / 32; ++i) s += s_warp[i];
+                atomicAdd(&P.out[P.t[cur].slot], s);
+            }
+            acc = 0.0;
+        }
+        if (!more) break;
+        cur = t;
+        const NormDesc& d = P.t[t];
+        const char* base = (const char*)d.base16;
+        const int64_t lo = d.lead_f32 & 0xff;
+        const bool f32 = (d.lead_f32 >> 8) != 0;
+        const int64_t hi = d.span_bytes;
+        const int64_t item_off = (int64_t)(w - item_begin) * kNormItemBytes;
+#pragma unroll
+        for (int k = 0; k < kNormVecPerThread; ++k) {
+            const int64_t off = item_off + (int64_t)(k * kNormThreads + tid) * 16;
+            if (off >= lo && off + 16 <= hi) {
+                const uint4 v = ld_stream16(base + off);
+                acc = f32 ? acc + sq4_f32(v) : sq8_bf16(v, acc);
+            } else if (off + 16 > lo && off < hi) {
+                acc += sq_partial(base, off, lo, hi, f32);
+            }
+        }
+    }
+}
+
+__global__ void skip_count_kernel(const double* sqnorm, int32_t* count) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) *count = isfinite(*sqnorm) ? 0 : *count + 1;
+}
+
+}  // namespace lt
+
+extern "C" int lt_grad_sqnorm_per_tensor(const lt_tensor* tensors, int32_t n, double* d_out, lt_stream stream) {
+    using namespace lt;
+    if (n < 0 || (n > 0 && tensors == nullptr) || (n > 0 && d_out == nullptr)) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_out & 7) != 0) return LT_ERR_ALIGNMENT;
+    for (int32_t i = 0; i < n; ++i) {
+        const lt_tensor& x = tensors[i];
+        if (x.numel < 0) return LT_ERR_INVALID_ARG;
+        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;
+        if (x.numel == 0) continue;
+        if ((x.grad_dtype != LT_F32 && x.grad_dtype != LT_BF16) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
+        if (((uintptr_t)x.grad % (x.grad_dtype == LT_F32 ? 4 : 2)) != 0) return LT_ERR_ALIGNMENT;
+    }
+    DeviceInfo* dev = nullptr;
+    int rc = ensure_device((cudaStream_t)stream, &dev);
+    if (rc != LT_OK) return rc;
+    NormParams P;
+    P.ticket = nullptr; P.partials = nullptr; P.out = d_out;
+    int32_t i = 0;
+    while (i < n) {
+        int cnt = 0;
+        int64_t items = 0;
+        while (i < n && cnt < kCap) {
+            const lt_tensor& x = tensors[i];
+            if (x.numel == 0) { ++i; continue; }
+            const uintptr_t a = (uintptr_t)x.grad;
+            const int lead = (int)(a & 15);
+            const int64_t span = lead + x.numel * (x.grad_dtype == LT_F32 ? 4 : 2);
+            const int64_t it = (span + kNormItemBytes - 1) / kNormItemBytes;
+            if (items + it > 0x7fffffff) break;
+            NormDesc& d = P.t[cnt];
+            d.base16 = (const void*)(a - lead);
+            d.span_bytes = span;
+            items += it;
+            d.item_end = (int32_t)items;
+            d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
+            d.slot = i;
+            ++cnt; ++i;
+        }
+        if (cnt == 0) continue;
+        P.n = cnt;
+        P.total_items = (int32_t)items;
+        int grid = kNormCtasPerSm * dev->sm_count;
+        if (grid > P.total_items) grid = P.total_items;
+        sqnorm_per_tensor_kernel<<<grid, kNormThreads, 0, (cudaStream_t)stream>>>(P);
+        if (cudaGetLastError() != cudaSuccess) return LT_ERR_CUDA;
+    }
+    return LT_OK;
+}
+
+extern "C" int lt_skip_count_update(const double* d_sqnorm, int32_t* d_skip_count, lt_stream stream) {
+    if (!d_sqnorm || !d_skip_count) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_sqnorm & 7) != 0 || ((uintptr_t)d_skip_count & 3) != 0) return LT_ERR_ALIGNMENT;
+    lt::skip_count_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_sqnorm, d_skip_count);
+    return cudaGetLastError() == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
+
 // ---- lt_grad_sqnorm_multi_noalloc ------------------------------------------------------------------
 // Same kernel, scratch in a module-scope device array instead of a caller-supplied workspace.
 namespace {

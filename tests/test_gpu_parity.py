@@ -275,3 +275,32 @@ def test_hybrid_decoder_split_matches_target_fraction():
     n8 = sum(s for s, f in zip(spec.sizes, spec.state_f32) if not f)
     assert 0.015 <= n8 / spec.numel <= 0.03
     run_free(spec, 4096, 2, check_every_step=False)
+
+
+def test_per_tensor_norms_and_skip_counter():
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=700, max_numel=1 << 17, seed=19)      # more tensors than one launch holds
+    buf = W.Buffers(spec, 2048, DEV)
+    W.fill_params(buf); W.fill_grads(buf, 1)
+    tl = L.TensorList.from_buffers(buf)
+    out = torch.zeros(tl.n, dtype=torch.float64, device=DEV)
+    L.lt_grad_sqnorm_per_tensor(tl, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    ots, _ = oracle_tensors(buf)
+    ref = np.array([O.sqnorm([t]) for t in ots])
+    assert np.all(np.abs(got - ref) <= 1e-12 * np.maximum(ref, 1e-300))
+    assert np.all(got[ref == 0] == 0)                                      # the all-zero-gradient tensors
+    assert abs(got.sum() - O.sqnorm(ots)) <= 1e-11 * ref.sum()
+    # consecutive non-finite steps are counted on the device and reset by a finite one
+    opt = L.Hybrid8Optimizer(tl, 2048, L.HParams(max_norm=0.5))
+    opt.init_state()
+    seen = []
+    for k, bad in enumerate([False, True, True, False, True, True, True], start=1):
+        W.fill_grads(buf, k)
+        if bad:
+            buf.view("grad", 5)[0] = float("inf")
+        opt.step()
+        seen.append(int(opt.skip_count.item()))
+    assert seen == [0, 1, 2, 0, 1, 2, 3]
+    assert int(opt.status.item()) & 1
