@@ -259,6 +259,43 @@ def time_e2e(name, block, steps, warmup):
     return out
 
 
+def time_host_resident(name, block, steps):
+    """The paper's own layout: parameters, gradients and state in pinned HOST memory, streamed through
+    the kernels in layer-group chunks (paper_2608_11919_b200/host_resident.py); everything crosses the host
+    link every step, in both directions."""
+    import torch
+    import paper_2608_11919_b200 as L
+    from paper_2608_11919_b200 import workloads as W
+    from paper_2608_11919_b200.host_resident import HostResidentOptimizer
+    dev = torch.device("cuda", torch.cuda.current_device())
+    spec = W.SPECS[name]()
+    host = W.Buffers(spec, block, "cpu", pin=True)
+    tmp = W.Buffers(spec, block, dev)               # generate on the device, copy out, free
+    W.fill_params(tmp); W.fill_grads(tmp, 1)
+    host.param.copy_(tmp.param); host.grad.copy_(tmp.grad)
+    del tmp
+    torch.cuda.empty_cache()
+    opt = HostResidentOptimizer(host, block, L.HParams(max_norm=spec.max_norm), W.layer_groups(spec, 4), device=dev)
+    opt.init_state()
+    opt.step()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        opt.step()
+    end.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(end) / steps
+    out = {"workload": name, "value": spec.numel / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+           "h2d_bytes_per_step": int(opt.h2d_bytes), "d2h_bytes_per_step": int(opt.d2h_bytes),
+           "h2d_gbs": opt.h2d_bytes / (ms * 1e-3) / 1e9, "status": float(opt.result[1]),
+           "what": "parameters, gradients and 8-bit state resident in pinned host memory; all of it copied in and the "
+                   "updated parameters and state copied out every step, overlapped with the kernels"}
+    del opt, host
+    torch.cuda.empty_cache()
+    return out
+
+
 def oracle_sample_time(name: str, block: int, target_params: int):
     """Times the CPU oracle (norm + step, one thread) on the first tensors/blocks of the workload,
     with the workload's value recipe generated on the host. Returns (params/s, sample description)."""
@@ -307,6 +344,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-alt-block", action="store_true", help="skip the second run at the other block size")
+    ap.add_argument("--host-resident", default="3b", help="workload of the host-resident end-to-end run, or 'none'")
     ap.add_argument("--cpu-sample", type=int, default=128 << 20, help="params in the oracle's timed sample")
     args = ap.parse_args()
 
@@ -381,6 +419,12 @@ def main():
             e2e["value"] = h["params"] * world / (e2e["ms_per_step"] * 1e-3)
             e2e["h2d_bytes_per_step"] *= world
             e2e["d2h_bytes_per_step"] *= world
+    host_state = None
+    if not args.no_e2e and not dist_on and args.host_resident != "none":
+        try:
+            host_state = time_host_resident(args.host_resident, args.block, 3)
+        except (RuntimeError, MemoryError) as e:      # e.g. the host refuses to pin that much memory
+            host_state = {"workload": args.host_resident, "skipped": str(e)[:120]}
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, desc, dt = oracle_sample_time(head, args.block, args.cpu_sample)
@@ -409,7 +453,7 @@ def main():
                            "parallelism": f"shard{world}+scalar-allreduce" if world > 1 else "single"},
                 "roofline": roof, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": h["launches_per_step"] * args.steps, "clocks": h["clocks"],
-                "other_block": alt, "workloads": results, "notes": notes}
+                "other_block": alt, "e2e_host_resident": host_state, "workloads": results, "notes": notes}
         print(json.dumps(line))
     if dist_on:
         torch.distributed.destroy_process_group()
