@@ -125,7 +125,10 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
 
 template <bool PRECISE, bool P_BF16>
 int launch(const StepParams& p, int sm_count, cudaStream_t s) {
-    static int full_grid = 0;
+    static int grid_of_device[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return LT_ERR_CUDA; }
+    int& full_grid = grid_of_device[dev];
     if (full_grid == 0) {
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adamw32_kernel<PRECISE, P_BF16>, kNT, 0) != cudaSuccess ||

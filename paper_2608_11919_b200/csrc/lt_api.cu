@@ -119,11 +119,11 @@ const uint32_t* host_lut(bool is_signed, bool full) {
 
 // ---- per-device set-up ---------------------------------------------------------------------------
 static std::mutex g_mu;
-static DeviceInfo g_dev[64];
+static DeviceInfo g_dev[kMaxDevices];
 
 int ensure_device(cudaStream_t stream, DeviceInfo** out) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LT_ERR_CUDA; }
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return LT_ERR_CUDA; }
     std::lock_guard<std::mutex> lock(g_mu);
     DeviceInfo& d = g_dev[dev];
     if (!d.tables_ready) {

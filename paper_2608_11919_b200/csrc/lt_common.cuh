@@ -11,6 +11,7 @@ namespace lt {
 // Tensors per launch: descriptors travel as kernel parameters (no device table, no copy to keep
 // alive), and the parameter space of sm_100 holds 32764 bytes.
 constexpr int kCap = 480;
+constexpr int kMaxDevices = 64;   // device ordinals the per-device caches cover
 
 constexpr int kFlagParamBf16 = 1;
 constexpr int kFlagGradF32 = 2;
