@@ -114,3 +114,39 @@ def test_ragged_full_ten_steps_sampled_tensors():
         st.check()
     print("ragged full:", spec.numel, "elements,", len(chosen), "tensors compared", st)
     assert int(opt.status.item()) == 0
+
+
+def test_single_tensor_beyond_two_to_the_31_elements():
+    """Index arithmetic at the top of the range: one tensor of 2^31 + 6161 elements (8.6 GB of fp32
+    parameters, a ragged last block), compared on blocks at the start, around the 2^30 / 2^31 element marks
+    (the 2^32-byte marks of the fp32 and bf16 arrays and the 2^31-byte mark of the code arrays) and at the end."""
+    torch.cuda.set_device(0)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24e9:
+        pytest.skip("needs 24 GB of device memory")
+    block = 2048
+    n = (1 << 31) + 3 * block + 17
+    spec = W.Spec("huge", ["w"], [n], [-1], torch.float32, seed=31, grad_std=1e-4, grad_kind="normal",
+                  max_norm=1.0, steps=1, align_elems=16)
+    buf = W.Buffers(spec, block, "cuda:0")
+    W.fill_params(buf)
+    tl = L.TensorList.from_buffers(buf)
+    opt = L.Hybrid8Optimizer(tl, block, L.HParams(max_norm=1.0))
+    opt.init_state()
+    for k in (1, 2):
+        W.fill_grads(buf, k)
+        opt.step()
+    nb = (n + block - 1) // block
+    marks = [0, (1 << 30) // block - 1, (1 << 31) // block - 2, nb - 3]
+    slices = [(0, b, 3) for b in marks]
+    W.fill_grads(buf, 3)
+    ots, slices = oracle_tensors(buf, slices=slices)
+    opt.step()
+    torch.cuda.synchronize()
+    S_gpu, S = float(opt.sqnorm.item()), oracle_sqnorm_of_buffers(buf)
+    assert abs(S_gpu - S) <= NORM_RTOL * S
+    assert parallel_oracle_step(ots, block, O.HParams(max_norm=1.0, step=3), S) == 0
+    st = compare(buf, ots, slices)
+    print("huge tensor:", st)
+    st.check()
+    assert ots[-1].numel == 2 * block + 17                      # the ragged tail was among the compared blocks
