@@ -114,7 +114,9 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  * If S is NaN or Inf nothing is written except bit 0 of *d_status (the paper's "non-finite gradients
  * are skipped", training-configuration table); the caller clears d_status when it wants to.
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
- * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). */
+ * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). The parameter
+ * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-15 or, for bf16
+ * parameters, a step size lr / (1 - beta1^t) above 1e-4, where it is IEEE-exact as well. */
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 

@@ -340,12 +340,17 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
     P.s.max_norm = hp->max_norm;
     P.s.clip_on = clip_on ? 1 : 0;
     // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps
-    P.s.precise_param = (hp->eps < 1e-15f) ? 1 : 0;
+    const bool precise_any = hp->eps < 1e-15f;
+    // Large steps into bf16 parameters also take the exact path: the approximate one is off by ~3e-7 of the
+    // update, which shows after rounding to bf16 once the update is not tiny against the parameter's ulp
+    // (and without bound where update and parameter cancel).
+    const bool precise_bf16 = precise_any || P.s.step_size > 1e-4f;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
     for (int st = LT_STATE_U8; st <= LT_STATE_F32; ++st) {
         for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype and one state kind per launch
             P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
+            P.s.precise_param = (dt == LT_BF16 ? precise_bf16 : precise_any) ? 1 : 0;
             int32_t i = 0;
             while (i < n) {
                 pack_step(tensors, n, st == LT_STATE_F32 ? kAdamw32Item : block, &i, &P, true, dt, st);

@@ -304,3 +304,38 @@ def test_per_tensor_norms_and_skip_counter():
         seen.append(int(opt.skip_count.item()))
     assert seen == [0, 1, 2, 0, 1, 2, 3]
     assert int(opt.status.item()) & 1
+
+
+@pytest.mark.parametrize("hp_kw", [
+    dict(eps=0.0),                                   # tiny eps: the kernel takes IEEE sqrt and divide for the parameter
+    dict(eps=1e-20, lr=1e-3),
+    dict(beta1=0.0, beta2=0.5, weight_decay=0.0, lr=1e-2),
+    dict(beta1=0.99, beta2=0.9999, eps=1e-6, lr=3e-4, weight_decay=0.1),
+])
+def test_other_hyper_parameters(hp_kw):
+    for pd in (torch.float32, torch.bfloat16):
+        spec = W.ragged_spec(n_tensors=80, max_numel=1 << 15, seed=23)
+        spec.param_dtype = pd
+        spec.zero_grad_frac = 0.0 if hp_kw.get("eps", 1.0) == 0.0 else spec.zero_grad_frac   # 0/0 is nobody's parity case
+        run_free(spec, 2048, 3, hp_kw=hp_kw)
+
+
+def test_late_step_count_and_infinite_max_norm():
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=60, max_numel=1 << 15, seed=24)
+    buf = W.Buffers(spec, 4096, DEV)
+    W.fill_params(buf); W.fill_grads(buf, 1)
+    tl = L.TensorList.from_buffers(buf)
+    L.lt_hybrid8_state_init(tl, 4096)
+    ots, slices = oracle_tensors(buf)
+    sq = torch.zeros(1, dtype=torch.float64, device=DEV)
+    ws = torch.empty(L.lt_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    for t in (1000, 100000):                         # bias corrections ~1
+        W.fill_grads(buf, t)
+        refresh_grads(ots, buf, slices)
+        sq.zero_()
+        L.lt_grad_sqnorm_multi(tl, sq, ws)
+        L.lt_hybrid8_step(tl, 4096, L.HParams(max_norm=float("inf"), step=t), sq, None)
+        torch.cuda.synchronize()
+        O.hybrid8_step(ots, 4096, O.HParams(max_norm=float("inf"), step=t), O.sqnorm(ots))
+        compare(buf, ots, slices).check()
