@@ -339,3 +339,53 @@ def test_late_step_count_and_infinite_max_norm():
         torch.cuda.synchronize()
         O.hybrid8_step(ots, 4096, O.HParams(max_norm=float("inf"), step=t), O.sqnorm(ots))
         compare(buf, ots, slices).check()
+
+
+def test_empty_lists_and_empty_tensors():
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=12, max_numel=1 << 13, seed=25)
+    buf = W.Buffers(spec, 2048, DEV)
+    W.fill_params(buf); W.fill_grads(buf, 1)
+    views = {k: [buf.view(k, t) for t in range(12)] for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax")}
+    for k in views:                                   # tensors 2 and 7 become empty
+        for t in (2, 7):
+            views[k][t] = views[k][t][:0]
+    tl = L.TensorList(*[views[k] for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax")])
+    full = L.TensorList.from_buffers(buf, [t for t in range(12) if t not in (2, 7)])
+    ws = torch.empty(L.lt_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    a = torch.zeros(1, dtype=torch.float64, device=DEV); b = torch.zeros(1, dtype=torch.float64, device=DEV)
+    L.lt_hybrid8_state_init(tl, 2048)
+    L.lt_grad_sqnorm_multi(tl, a, ws); L.lt_grad_sqnorm_multi(full, b, ws)
+    L.lt_grad_sqnorm_multi(tl.slice(0, 0), a, ws)     # an empty list is a no-op
+    L.lt_hybrid8_step(tl.slice(0, 0), 2048, L.HParams(), a, None)
+    before = buf.param.clone()
+    L.lt_hybrid8_step(tl, 2048, L.HParams(), a, None)
+    torch.cuda.synchronize()
+    assert float(a.item()) == float(b.item()) > 0
+    for t in range(12):
+        changed = not torch.equal(buf.view("param", t), before[buf.off[t]: buf.off[t] + spec.sizes[t]])
+        assert changed == (t not in (2, 7)), t         # the emptied tensors' storage was not touched
+
+
+def test_overflowing_moments_do_not_fault():
+    # clipping disabled and absurd gradients: v' overflows to +inf, the block maximum is inf, the normalised
+    # values are NaN. Nothing sensible can come out, but every table index stays in range, nothing faults,
+    # and the next ordinary step runs.
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=20, max_numel=1 << 14, seed=26)
+    for pd in (torch.float32, torch.bfloat16):
+        spec.param_dtype = pd
+        buf = W.Buffers(spec, 2048, DEV)
+        W.fill_params(buf)
+        tl = L.TensorList.from_buffers(buf)
+        opt = L.Hybrid8Optimizer(tl, 2048, L.HParams(max_norm=0.0))
+        opt.init_state()
+        buf.grad.fill_(1e30)
+        opt.step()
+        torch.cuda.synchronize()
+        assert int(opt.status.item()) == 0
+        opt.init_state()
+        W.fill_grads(buf, 1)
+        opt.step()
+        torch.cuda.synchronize()
+        assert bool(torch.isfinite(buf.m_absmax).all()) and bool(torch.isfinite(buf.param.float()).all())
