@@ -135,6 +135,28 @@ int lt_grad_sqnorm_per_tensor(const lt_tensor* tensors, int32_t n, double* d_out
  * aborts. One thread of device work. */
 int lt_skip_count_update(const double* d_sqnorm, int32_t* d_skip_count, lt_stream stream);
 
+/* Step count and the two step-dependent scalars, resident on the DEVICE, so that a whole optimizer step
+ * (norm, bookkeeping, update) can be recorded once in a CUDA graph and replayed every step with no host
+ * arithmetic in between. (No counterpart in the paper, whose optimizer runs on the host.) The caller
+ * allocates one lt_step_state on the device and zeroes it (step 0). */
+typedef struct {
+    int64_t step;          /* steps taken so far; lt_step_state_advance adds one          */
+    float step_size;       /* lr / (1 - beta1^step)                                       */
+    float inv_sqrt_bc2;    /* 1 / sqrt(1 - beta2^step)                                    */
+} lt_step_state;
+
+/* One thread of device work: d_state->step += 1, then step_size and inv_sqrt_bc2 for the new count from
+ * hp->lr, hp->beta1, hp->beta2 (formed in fp64, rounded once to fp32, like the host path; the device's
+ * fp64 pow may differ from the host's in the last bit, which can move step_size by one fp32 ulp). */
+int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, lt_stream stream);
+
+/* lt_hybrid8_step with the step count taken from the device: identical except that hp->step is ignored
+ * and step_size / inv_sqrt_bc2 are read from *d_state by the kernels. bf16 parameters take the exact
+ * parameter path when lr / (1 - beta1) > 1e-4 (the largest step size any count can give). */
+int lt_hybrid8_step_graph(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
+                          const lt_step_state* d_state, const double* d_sqnorm, int32_t* d_status,
+                          lt_stream stream);
+
 /* Largest number of non-empty tensors one lt_grad_sqnorm_multi_noalloc call accepts. */
 #define LT_NOALLOC_MAX_TENSORS 480
 

@@ -10,7 +10,7 @@ _BINDING_NAMES = (
     "LT_F32", "LT_BF16", "LtError", "HParams", "TensorList", "library_path",
     "lt_hybrid8_state_bytes", "lt_hybrid8_code_table", "lt_workspace_bytes", "lt_hybrid8_state_init",
     "lt_grad_sqnorm_multi", "lt_grad_sqnorm_multi_noalloc", "lt_grad_sqnorm_per_tensor", "lt_skip_count_update", "lt_hybrid8_step", "lt_status_str",
-    "Hybrid8Optimizer",
+    "Hybrid8Optimizer", "GraphedHybrid8Optimizer", "lt_step_state_advance", "lt_hybrid8_step_graph",
 )
 __all__ = list(_BINDING_NAMES)
 

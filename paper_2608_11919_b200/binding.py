@@ -55,6 +55,9 @@ def _load():
     L.lt_grad_sqnorm_multi_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.lt_grad_sqnorm_per_tensor.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.lt_skip_count_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.lt_step_state_advance.argtypes = [C.c_void_p, C.POINTER(_LtHParams), C.c_void_p]
+    L.lt_hybrid8_step_graph.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_LtHParams), C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p]
     return L
 
 
@@ -190,6 +193,62 @@ def lt_hybrid8_step(tensors: TensorList, block: int, hp: HParams, d_sqnorm: Opti
            _lib.lt_hybrid8_step(tensors.ptr, tensors.n, block, C.byref(h),
                                 None if d_sqnorm is None else d_sqnorm.data_ptr(),
                                 None if d_status is None else d_status.data_ptr(), _stream(stream)))
+
+
+def lt_step_state_advance(d_state: torch.Tensor, hp: HParams, stream=None) -> None:
+    """d_state: 16 bytes of device memory (an lt_step_state), zeroed once by the caller."""
+    assert d_state.is_cuda and d_state.numel() * d_state.element_size() >= 16
+    h = hp.c()
+    _check("lt_step_state_advance", _lib.lt_step_state_advance(d_state.data_ptr(), C.byref(h), _stream(stream)))
+
+
+def lt_hybrid8_step_graph(tensors: TensorList, block: int, hp: HParams, d_state: torch.Tensor,
+                          d_sqnorm: Optional[torch.Tensor], d_status: Optional[torch.Tensor], stream=None) -> None:
+    h = hp.c()
+    _check("lt_hybrid8_step_graph",
+           _lib.lt_hybrid8_step_graph(tensors.ptr, tensors.n, block, C.byref(h), d_state.data_ptr(),
+                                      None if d_sqnorm is None else d_sqnorm.data_ptr(),
+                                      None if d_status is None else d_status.data_ptr(), _stream(stream)))
+
+
+class GraphedHybrid8Optimizer:
+    """The whole optimizer step recorded once in a CUDA graph and replayed: zero the norm, norm over all
+    chunks, skip bookkeeping, advance the device-resident step state, update all chunks. Between replays the
+    caller only writes new gradients into the same buffers."""
+
+    def __init__(self, tensors: TensorList, block: int, hp: HParams, chunks: Optional[Sequence[TensorList]] = None,
+                 device=None):
+        device = device if device is not None else tensors._keep[0][0].device
+        self.tensors, self.block, self.hp = tensors, block, hp
+        self.chunks = list(chunks) if chunks is not None else [tensors]
+        self.sqnorm = torch.zeros(1, dtype=torch.float64, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.skip_count = torch.zeros(1, dtype=torch.int32, device=device)
+        self.state = torch.zeros(2, dtype=torch.int64, device=device)       # an lt_step_state, step 0
+        self.workspace = torch.empty(lt_workspace_bytes(), dtype=torch.uint8, device=device)
+        self.graph = None
+
+    def init_state(self) -> None:
+        lt_hybrid8_state_init(self.tensors, self.block)
+
+    def _enqueue(self) -> None:
+        self.sqnorm.zero_()
+        for ch in self.chunks:
+            lt_grad_sqnorm_multi(ch, self.sqnorm, self.workspace)
+        lt_skip_count_update(self.sqnorm, self.skip_count)
+        lt_step_state_advance(self.state, self.hp)
+        for ch in self.chunks:
+            lt_hybrid8_step_graph(ch, self.block, self.hp, self.state, self.sqnorm, self.status)
+
+    def step(self) -> None:
+        if self.graph is None:
+            self._enqueue()                      # first step eagerly: one-time set-up must not be captured
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self._enqueue()
+            self.graph = g
+            return
+        self.graph.replay()
 
 
 class Hybrid8Optimizer:

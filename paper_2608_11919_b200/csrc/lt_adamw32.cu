@@ -52,6 +52,7 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
     }
     r.beta1 = P.s.beta1; r.beta2 = P.s.beta2; r.omb1 = P.s.omb1; r.omb2 = P.s.omb2;
     r.step_size = P.s.step_size; r.isb2 = P.s.inv_sqrt_bc2; r.decay = P.s.decay; r.eps = P.s.eps;
+    if (P.dev_scalars != nullptr) { r.step_size = P.dev_scalars[0]; r.isb2 = P.dev_scalars[1]; }
 
     int t = 0, begin = 0;
     for (int w = blockIdx.x; w < P.total_blocks; w += gridDim.x) {
@@ -141,6 +142,21 @@ int launch(const StepParams& p, int sm_count, cudaStream_t s) {
 }
 
 }  // namespace
+
+__global__ void step_state_advance_kernel(lt_step_state* st, float lr, float beta1, float beta2) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const int64_t t = st->step + 1;
+    const double bc1 = 1.0 - pow((double)beta1, (double)t);
+    const double bc2 = 1.0 - pow((double)beta2, (double)t);
+    st->step = t;
+    st->step_size = (float)((double)lr / bc1);
+    st->inv_sqrt_bc2 = (float)(1.0 / sqrt(bc2));
+}
+
+int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, cudaStream_t s) {
+    step_state_advance_kernel<<<1, 32, 0, s>>>(d_state, lr, beta1, beta2);
+    return cudaGetLastError() == cudaSuccess ? LT_OK : LT_ERR_CUDA;
+}
 
 int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s) {
     if (p.param_bf16) return p.s.precise_param ? launch<true, true>(p, sm_count, s) : launch<false, true>(p, sm_count, s);

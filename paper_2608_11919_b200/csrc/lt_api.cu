@@ -257,7 +257,7 @@ int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt
     if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
     StepParams P;
     std::memset(&P.s, 0, sizeof(P.s));
-    P.sqnorm = nullptr; P.status = nullptr; P.param_bf16 = 0;
+    P.sqnorm = nullptr; P.status = nullptr; P.param_bf16 = 0; P.dev_scalars = nullptr;
     int32_t i = 0;
     while (i < n) {
         pack_step(tensors, n, block, &i, &P, false, -1);
@@ -311,10 +311,18 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
     return LT_OK;
 }
 
-int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
-                    const double* d_sqnorm, int32_t* d_status, lt_stream stream) {
+static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp_in,
+                     const lt_step_state* d_state, bool use_state, const double* d_sqnorm, int32_t* d_status,
+                     lt_stream stream) {
     if (!valid_block(block)) return LT_ERR_UNSUPPORTED;
-    if (!hp) return LT_ERR_INVALID_ARG;
+    if (!hp_in) return LT_ERR_INVALID_ARG;
+    lt_hparams hp_local = *hp_in;
+    if (use_state) {
+        if (!d_state) return LT_ERR_INVALID_ARG;
+        if (!aligned(d_state, 8)) return LT_ERR_ALIGNMENT;
+        hp_local.step = 1;   // the largest step size any count can give; the kernels read the real scalars
+    }
+    const lt_hparams* hp = &hp_local;
     int rc = validate_tensors(tensors, n, NEED_GRAD | NEED_PARAM | NEED_STATE);
     if (rc != LT_OK) return rc;
     if (hp->step < 1 || !(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) ||
@@ -347,6 +355,7 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
     const bool precise_bf16 = precise_any || P.s.step_size > 1e-4f;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
+    P.dev_scalars = use_state ? &d_state->step_size : nullptr;
     for (int st = LT_STATE_U8; st <= LT_STATE_F32; ++st) {
         for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype and one state kind per launch
             P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
@@ -362,6 +371,25 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
         }
     }
     return LT_OK;
+}
+
+int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
+                    const double* d_sqnorm, int32_t* d_status, lt_stream stream) {
+    return step_impl(tensors, n, block, hp, nullptr, false, d_sqnorm, d_status, stream);
+}
+
+int lt_hybrid8_step_graph(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
+                          const lt_step_state* d_state, const double* d_sqnorm, int32_t* d_status,
+                          lt_stream stream) {
+    return step_impl(tensors, n, block, hp, d_state, true, d_sqnorm, d_status, stream);
+}
+
+int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, lt_stream stream) {
+    if (!d_state || !hp) return LT_ERR_INVALID_ARG;
+    if (!aligned(d_state, 8)) return LT_ERR_ALIGNMENT;
+    if (!(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) || !std::isfinite(hp->lr))
+        return LT_ERR_INVALID_ARG;
+    return launch_step_state_advance(d_state, hp->lr, hp->beta1, hp->beta2, (cudaStream_t)stream);
 }
 
 }  // extern "C"

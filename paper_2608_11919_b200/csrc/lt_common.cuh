@@ -50,6 +50,7 @@ struct StepParams {
     StepScalars s;
     const double* sqnorm;
     int32_t* status;
+    const float* dev_scalars;   // non-null: {step_size, inv_sqrt_bc2} are read from the device (lt_step_state)
     int32_t n;
     int32_t total_blocks;
     int32_t param_bf16;         // parameter dtype of every tensor of this launch
@@ -91,6 +92,7 @@ int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s);   // tensors with fp32 moments
 constexpr int kAdamw32Item = 2048;   // elements per work item of that kernel (items restart at every tensor)
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
+int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, cudaStream_t s);
 int upload_tables(cudaStream_t s);
 
 #ifndef LT_NORM_THREADS
