@@ -389,3 +389,19 @@ def test_overflowing_moments_do_not_fault():
         opt.step()
         torch.cuda.synchronize()
         assert bool(torch.isfinite(buf.m_absmax).all()) and bool(torch.isfinite(buf.param.float()).all())
+
+
+def test_gpu_norm_against_exact_sum():
+    # the kernel adds exact fp64 squares; against the exactly rounded sum (math.fsum) it is far more accurate
+    # than the 1e-5 tolerance asks for, and more accurate than one long sequential fp64 sum
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=300, max_numel=1 << 16, seed=27)
+    buf = W.Buffers(spec, 2048, DEV)
+    W.fill_grads(buf, 1)
+    tl = L.TensorList.from_buffers(buf)
+    acc = torch.zeros(1, dtype=torch.float64, device=DEV)
+    ws = torch.empty(L.lt_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    L.lt_grad_sqnorm_multi(tl, acc, ws)
+    g = buf.grad[:buf.total].float().double().cpu().numpy()
+    exact = math.fsum((g * g).tolist())
+    assert abs(float(acc.item()) - exact) <= 1e-13 * exact
