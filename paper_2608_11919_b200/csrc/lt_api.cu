@@ -203,7 +203,19 @@ static void pack_step(const lt_tensor* t, int32_t n, int32_t block, int32_t* i, 
         if (with_pg) {
             if (x.param_dtype == LT_BF16) flags |= kFlagParamBf16;
             if (x.grad_dtype == LT_F32) flags |= kFlagGradF32;
-            vec = vec && aligned(x.param, 4 * esize(x.param_dtype)) && aligned(x.grad, 4 * esize(x.grad_dtype));
+            const int ps = esize(x.param_dtype), gs = esize(x.grad_dtype);
+            vec = vec && aligned(x.param, 4 * ps) && aligned(x.grad, 4 * gs);
+            if (!vec && !st32) {
+                // tensors packed back to back: skipping `sh` elements may align all four arrays at once
+                for (int sh = 1; sh < 4; ++sh) {
+                    if (aligned((const char*)x.param + sh * ps, 4 * ps) && aligned((const char*)x.grad + sh * gs, 4 * gs) &&
+                        aligned(x.m_code + sh, 4) && aligned(x.v_code + sh, 4)) {
+                        vec = true;
+                        flags |= sh << kFlagShiftPos;
+                        break;
+                    }
+                }
+            }
         }
         if (vec) flags |= kFlagVecOk;
         if (with_pg && aligned(x.param, 16) && aligned(x.grad, 16) && aligned(x.m_code, 16) && aligned(x.v_code, 16))

@@ -15,8 +15,9 @@ constexpr int kMaxDevices = 64;   // device ordinals the per-device caches cover
 
 constexpr int kFlagParamBf16 = 1;
 constexpr int kFlagGradF32 = 2;
-constexpr int kFlagVecOk = 4;   // every pointer allows 4-element vector access
+constexpr int kFlagVecOk = 4;   // every pointer allows 4-element vector access (after the common shift, if any)
 constexpr int kFlagStateF32 = 16; // moments are plain fp32 arrays (mc / vc point to float)
+constexpr int kFlagShiftPos = 8;  // bits 8-9: elements to skip until all four arrays are vector-aligned together
 constexpr int kFlagBulkOk = 8;  // every pointer is 16-byte aligned (bulk prefetch of whole blocks allowed)
 
 struct StepDesc {               // 64 bytes
