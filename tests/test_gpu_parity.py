@@ -405,3 +405,12 @@ def test_gpu_norm_against_exact_sum():
     g = buf.grad[:buf.total].float().double().cpu().numpy()
     exact = math.fsum((g * g).tolist())
     assert abs(float(acc.item()) - exact) <= 1e-13 * exact
+
+
+@pytest.mark.parametrize("block", [256, 512, 1024, 8192, 16384])
+def test_aligned_tensors_at_every_other_block_size(block):
+    # 16-byte aligned tensors take the vector path with bulk L2 prefetch at every supported block size
+    for pd in (torch.float32, torch.bfloat16):
+        spec = W.tiny_spec()
+        spec.param_dtype = pd
+        run_free(spec, block, 2)
