@@ -37,7 +37,7 @@ struct HostTables {
         qu[255] = 1.0f;
         fill_mid(qs, mid_s);
         fill_mid(qu, mid_u);
-        lut_ok = build_lut(mid_u, 7, false, 128, lut_u_full) && build_lut(mid_s, 6, true, 128, lut_s_full) &&
+        lut_ok = build_lut(mid_u, 7, false, 128, lut_u_full) && build_lut(mid_s, 6, true, 128, lut_s_full, true) &&
                  build_lut(mid_u, 7, false, 32, lut_u_compact) && build_lut(mid_s, 6, true, 32, lut_s_compact);
     }
     static int code_of(const float* mid, float x) {   // number of thresholds strictly below x
@@ -59,10 +59,12 @@ struct HostTables {
     //   x <  0:  entry = ((base + 1) << 24 | frac(T)) + H;             sum = entry + ~a
     //            (= (base + 1) << 24 + frac(T) - frac(x) - 1, which keeps base + 1 exactly when
     //            frac(x) < frac(T), i.e. x > T; no T: frac(T) = 0)
+    //            With neg_adds_iabs the kernel adds |u|_int of the raw bits u instead (one instruction):
+    //            for u < 0, |u|_int = ~a - 0x7fffffff, so the entry carries + 0x7fffffff.
     // Unsigned map: 128 x 128 buckets. Signed map: 128 x 64 buckets of the magnitude, positive half
     // first, negative half second. Exponent fields 128..255 (|x| >= 2, Inf, NaN) cannot occur for a
     // normalised moment; the kernel masks the index so that even then the lookup stays inside the table.
-    static bool build_lut(const float* mid, int mbits, bool is_signed, int binades, uint32_t* lut) {
+    static bool build_lut(const float* mid, int mbits, bool is_signed, int binades, uint32_t* lut, bool neg_adds_iabs = false) {
         const int per_binade = 1 << mbits, half = binades * per_binade, fbits = 23 - mbits;
         const int e_first = 128 - binades;   // first exponent field covered
         const uint32_t fmask = (1u << fbits) - 1u;
@@ -86,7 +88,7 @@ struct HostTables {
                 if (h == 1 && ca + 1 > 255) return false;
                 uint32_t e;
                 if (h == 0) e = (((uint32_t)ca << 24) | (0xFFFFFFu - (has_t ? tf : fmask))) - lo;
-                else e = (((uint32_t)(ca + 1) << 24) | (has_t ? tf : 0u)) + lo;
+                else e = (((uint32_t)(ca + 1) << 24) | (has_t ? tf : 0u)) + lo + (neg_adds_iabs ? 0x7fffffffu : 0u);
                 lut[h * half + key] = e;
             }
         }
