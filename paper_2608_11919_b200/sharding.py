@@ -21,6 +21,46 @@ def partition_tensors(sizes: Sequence[int], world: int) -> List[List[int]]:
     return [sorted(x) for x in out]
 
 
+def partition_contiguous(sizes: Sequence[int], world: int) -> List[range]:
+    """Splits the tensor list into `world` consecutive runs of near-equal element counts (run r ends at
+    the tensor boundary closest to r+1 world-ths of the total; runs may be empty when there are fewer
+    tensors than ranks). With tensors packed back to back, each rank then owns ONE contiguous slice of
+    the flat parameter buffer, which is what `allgather_params` exchanges."""
+    assert world >= 1
+    total = sum(int(x) for x in sizes)
+    cum, acc = [0], 0
+    for x in sizes:
+        acc += int(x)
+        cum.append(acc)
+    cuts = [0]
+    for r in range(1, world):
+        target = total * r / world
+        j = min(range(cuts[-1], len(sizes) + 1), key=lambda k: (abs(cum[k] - target), k))
+        cuts.append(j)
+    cuts.append(len(sizes))
+    return [range(cuts[r], cuts[r + 1]) for r in range(world)]
+
+
+def allgather_params(param_flat: torch.Tensor, bounds: Sequence[Sequence[int]], group=None) -> None:
+    """For replicated parameters: after the step every rank has updated only the slice it owns;
+    `bounds[r] = (begin, end)` is rank r's element range of `param_flat`. Each slice is broadcast from
+    its owner into the same place on every other rank (each GPU receives into its own memory; plain
+    NCCL, no peer loads in any kernel of this library). Slices may be empty or of different lengths."""
+    if not (torch.distributed.is_available() and torch.distributed.is_initialized()):
+        return
+    world = torch.distributed.get_world_size(group)
+    if world == 1:
+        return
+    assert len(bounds) == world
+    work = []
+    for r, (a, b) in enumerate(bounds):
+        if b > a:
+            src = torch.distributed.get_global_rank(group, r) if group is not None else r
+            work.append(torch.distributed.broadcast(param_flat[a:b], src=src, group=group, async_op=True))
+    for w in work:
+        w.wait()
+
+
 def allreduce_sqnorm(sqnorm: torch.Tensor, group=None) -> None:
     """Sum the per-rank squared norms in place (one fp64 element). On CUDA tensors this is enqueued on
     the current stream by NCCL, so it sits between the norm and the step without a host sync."""

@@ -100,3 +100,59 @@ def test_two_ranks_reproduce_the_unsharded_step():
             for a, b in zip(arrs, ref):
                 assert np.array_equal(a, b)
     assert seen == set(range(len(spec.sizes)))
+
+
+def test_contiguous_partition_covers_in_order():
+    spec = W.ragged_spec(n_tensors=300, max_numel=1 << 16, seed=2)
+    total = sum(spec.sizes)
+    for world in (1, 2, 3, 8):
+        runs = S.partition_contiguous(spec.sizes, world)
+        assert [i for r in runs for i in r] == list(range(300))
+        loads = [sum(spec.sizes[i] for i in r) for r in runs]
+        assert max(abs(l - total / world) for l in loads) <= max(spec.sizes)
+    assert [len(r) for r in S.partition_contiguous([5, 5], 4)] in ([1, 0, 1, 0], [0, 1, 0, 1], [1, 0, 0, 1], [0, 1, 1, 0])
+    assert [list(r) for r in S.partition_contiguous([], 2)] == [[], []]
+
+
+def _gather_worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        spec = W.ragged_spec(n_tensors=24, max_numel=1 << 12, seed=11)
+        runs = S.partition_contiguous(spec.sizes, world)
+        buf, ts = _make(spec, 1)                                     # every rank holds all parameters
+        mine = [ts[i] for i in runs[rank]]
+        s = torch.tensor([O.sqnorm(mine)], dtype=torch.float64)
+        S.allreduce_sqnorm(s)
+        assert O.hybrid8_step(mine, BLOCK, O.HParams(max_norm=0.5), float(s.item())) == 0
+        for i in runs[rank]:                                         # write the owned slice back into the replica
+            buf.view("param", i).copy_(torch.from_numpy(ts[i].param))
+        ends = [(buf.off[r[0]], buf.off[r[-1]] + spec.sizes[r[-1]]) if len(r) else (0, 0) for r in runs]
+        S.allgather_params(buf.param, ends)
+        q.put((rank, float(s.item()), buf.param.numpy().copy()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_allgather_rebuilds_the_replicated_parameters():
+    world = 3
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_gather_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = [q.get(timeout=120) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    spec = W.ragged_spec(n_tensors=24, max_numel=1 << 12, seed=11)
+    buf, ts = _make(spec, 1)
+    O.hybrid8_step(ts, BLOCK, O.HParams(max_norm=0.5), results[0][1])
+    for i, t in enumerate(ts):
+        buf.view("param", i).copy_(torch.from_numpy(t.param))
+    want = buf.param.numpy()
+    for _, _, got in results:                                       # every replica equals the unsharded update
+        assert np.array_equal(got, want)
