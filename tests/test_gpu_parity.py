@@ -311,6 +311,9 @@ def test_per_tensor_norms_and_skip_counter():
     dict(eps=1e-20, lr=1e-3),
     dict(beta1=0.0, beta2=0.5, weight_decay=0.0, lr=1e-2),
     dict(beta1=0.99, beta2=0.9999, eps=1e-6, lr=3e-4, weight_decay=0.1),
+    dict(lr=0.0),                                    # zero step size: only the decay factor (1) touches the parameter
+    dict(lr=1e-37, weight_decay=0.0),                # eps / step_size leaves the fp32 range
+    dict(lr=1e-6, eps=1e3),                          # the denominator is all eps
 ])
 def test_other_hyper_parameters(hp_kw):
     for pd in (torch.float32, torch.bfloat16):
