@@ -125,6 +125,18 @@ def test_every_small_size_and_alignment():
         run_free(spec, block, 2)
 
 
+def test_bf16_parameters_at_every_multiple_of_four_offset():
+    # tensor sizes that are multiples of 4 but not of 8 or 16: packed back to back, the bases run through
+    # every 4-element offset, so full blocks meet the 8-element vector path (16-byte aligned arrays), the
+    # 4-element one (8-byte aligned) and, with the single odd size, the shifted one
+    for block in (2048, 4096, 8192):
+        sizes = [2 * block + 4, block + 12, 3 * block + 8, block + 4, 2 * block + 16, block + 20, 2 * block + 1,
+                 block + 28, 2 * block + 4, block]
+        spec = to_bf16_params(W.ragged_spec(n_tensors=len(sizes), seed=31))
+        spec.sizes = sizes
+        run_free(spec, block, 3)
+
+
 def test_fp32_gradients():
     spec = W.ragged_spec(n_tensors=50, max_numel=1 << 15, seed=11)
     spec.grad_dtype = torch.float32
