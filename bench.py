@@ -196,6 +196,9 @@ def time_resident(name, block, steps, warmup, rank, world, dist_on, sample_clock
         "whole_gbs": N * (nb + sb) / (total_ms / steps * 1e-3) / 1e9,
         "step_ms_min": min(step_ms), "norm_ms_min": min(norm_ms),
         "step_ms_median": statistics.median(step_ms), "norm_ms_median": statistics.median(norm_ms),
+        # burst against sustained (the board's power limit lowers the clocks after ~0.1 s of launches)
+        "step_ms_first3": statistics.mean(step_ms[:3]), "step_ms_late_median": statistics.median(step_ms[steps // 2:]),
+        "norm_ms_late_median": statistics.median(norm_ms[steps // 2:]),
         "bytes_per_param": nb + sb, "status": status,
         "launches_per_step": (2 + (1 if 0 < n32 < N else 0)) * n_chunks, "fp32_state_fraction": n32 / N,
         "clocks": clocks,
