@@ -19,7 +19,7 @@ namespace {
 constexpr int kNT = 256;
 constexpr int kK = kAdamw32Item / (4 * kNT);
 
-struct Regs { float c, beta1, beta2, omb1, omb2, step_size, isb2, decay, eps, k1, k2; };
+struct Regs { float c, beta1, beta2, omb1, omb2, step_size, isb2, decay, eps; };
 
 __device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 __device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
@@ -33,8 +33,8 @@ __device__ __forceinline__ float update(const Regs& r, float p, float g, float& 
         const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), r.isb2), r.eps);
         return __fsub_rn(__fmul_rn(p, r.decay), __fmul_rn(r.step_size, __fdiv_rn(m, den)));
     }
-    const float u = __fmul_rn(m, rcp_approx(__fmaf_rn(sqrt_approx(v), r.k1, r.k2)));
-    return __fmaf_rn(p, r.decay, -u);
+    const float den = __fmaf_rn(sqrt_approx(v), r.isb2, r.eps);
+    return __fmaf_rn(-r.step_size, __fmul_rn(m, rcp_approx(den)), __fmul_rn(p, r.decay));   // p * decay rounded first, as defined
 }
 
 template <bool PRECISE, bool P_BF16>
@@ -53,7 +53,6 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
     r.beta1 = P.s.beta1; r.beta2 = P.s.beta2; r.omb1 = P.s.omb1; r.omb2 = P.s.omb2;
     r.step_size = P.s.step_size; r.isb2 = P.s.inv_sqrt_bc2; r.decay = P.s.decay; r.eps = P.s.eps;
     if (P.dev_scalars != nullptr) { r.step_size = P.dev_scalars[0]; r.isb2 = P.dev_scalars[1]; }
-    fold_step_size(r.step_size, r.isb2, r.eps, r.k1, r.k2);
 
     int t = 0, begin = 0;
     for (int w = blockIdx.x; w < P.total_blocks; w += gridDim.x) {

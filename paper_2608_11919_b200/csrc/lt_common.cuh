@@ -108,17 +108,4 @@ constexpr int kNormItemBytes = kNormThreads * kNormVecPerThread * 16;
 constexpr int kNormMaxCtas = 1024;
 constexpr int64_t kWorkspaceBytes = 256 + kNormMaxCtas * 8;
 
-// Approximate parameter path (S4): the step size is folded into the denominator,
-//   p' = p * decay - m' / (sqrt(v') * k1 + k2),   k1 = inv_sqrt_bc2 / step_size,   k2 = eps / step_size,
-// which saves one multiply per element. A step size of zero, or one so small that a quotient leaves the
-// fp32 range, gives k1 = 0, k2 = 2^127: the flush-to-zero reciprocal of that is 0 and p' = p * decay.
-#ifdef __CUDACC__
-__device__ __forceinline__ void fold_step_size(float step_size, float isb2, float eps, float& k1, float& k2) {
-    k1 = __fdiv_rn(isb2, step_size);
-    k2 = __fdiv_rn(eps, step_size);
-    if (!(fabsf(k1) < 3.0e38f) || !(fabsf(k2) < 3.0e38f)) { k1 = 0.0f; k2 = 1.7014118e38f; }
-}
-#endif
-
-
 }  // namespace lt
