@@ -24,17 +24,26 @@ struct Regs { float c, beta1, beta2, omb1, omb2, step_size, isb2, decay, eps; };
 __device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 __device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 
-template <bool PRECISE>
+// The parameter update exactly as defined (IEEE sqrt and divide, one rounding per operation).
+__device__ __forceinline__ float param_exact(const Regs& r, float p, float m, float v) {
+    const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), r.isb2), r.eps);
+    return __fsub_rn(__fmul_rn(p, r.decay), __fmul_rn(r.step_size, __fdiv_rn(m, den)));
+}
+
+// One element. GUARD (bf16 parameters on the approximate path): when p * decay and the update cancel to below
+// 2^-11 of p * decay, the approximate update's error (~2^-21 of the update) would be worth more than one bf16
+// ulp of the tiny result; such elements (about 2 in 10^7) take the exact formula. Same rule as the step kernel.
+template <bool PRECISE, bool GUARD>
 __device__ __forceinline__ float update(const Regs& r, float p, float g, float& m, float& v) {
     const float gc = __fmul_rn(g, r.c);
     m = __fadd_rn(__fmul_rn(r.beta1, m), __fmul_rn(r.omb1, gc));
     v = __fadd_rn(__fmul_rn(r.beta2, v), __fmul_rn(r.omb2, __fmul_rn(gc, gc)));
-    if (PRECISE) {
-        const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), r.isb2), r.eps);
-        return __fsub_rn(__fmul_rn(p, r.decay), __fmul_rn(r.step_size, __fdiv_rn(m, den)));
-    }
+    if (PRECISE) return param_exact(r, p, m, v);
     const float den = __fmaf_rn(sqrt_approx(v), r.isb2, r.eps);
-    return __fmaf_rn(-r.step_size, __fmul_rn(m, rcp_approx(den)), __fmul_rn(p, r.decay));   // p * decay rounded first, as defined
+    const float pd = __fmul_rn(p, r.decay);                                        // rounded first, as defined
+    const float pn = __fmaf_rn(-r.step_size, __fmul_rn(m, rcp_approx(den)), pd);
+    if (GUARD && __fmaf_rn(fabsf(pn), 2048.0f, -fabsf(pd)) < 0.0f) return param_exact(r, p, m, v);
+    return pn;
 }
 
 template <bool PRECISE, bool P_BF16>
@@ -90,10 +99,10 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
                 }
                 g[0] = __uint_as_float(gr[k].x << 16); g[1] = __uint_as_float(gr[k].x & 0xffff0000u);
                 g[2] = __uint_as_float(gr[k].y << 16); g[3] = __uint_as_float(gr[k].y & 0xffff0000u);
-                pn[0] = update<PRECISE>(r, p[0], g[0], mr[k].x, vr[k].x);
-                pn[1] = update<PRECISE>(r, p[1], g[1], mr[k].y, vr[k].y);
-                pn[2] = update<PRECISE>(r, p[2], g[2], mr[k].z, vr[k].z);
-                pn[3] = update<PRECISE>(r, p[3], g[3], mr[k].w, vr[k].w);
+                pn[0] = update<PRECISE, P_BF16 && !PRECISE>(r, p[0], g[0], mr[k].x, vr[k].x);
+                pn[1] = update<PRECISE, P_BF16 && !PRECISE>(r, p[1], g[1], mr[k].y, vr[k].y);
+                pn[2] = update<PRECISE, P_BF16 && !PRECISE>(r, p[2], g[2], mr[k].z, vr[k].z);
+                pn[3] = update<PRECISE, P_BF16 && !PRECISE>(r, p[3], g[3], mr[k].w, vr[k].w);
                 if (P_BF16) {
                     const __nv_bfloat162 lo = __floats2bfloat162_rn(pn[0], pn[1]);
                     const __nv_bfloat162 hi = __floats2bfloat162_rn(pn[2], pn[3]);
@@ -114,7 +123,7 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
                 const float g = g_f32 ? *(const float*)(gp + e * 4)
                                       : __uint_as_float((uint32_t)*(const unsigned short*)(gp + e * 2) << 16);
                 float m = mp[e], v = vp[e];
-                const float pn = update<PRECISE>(r, p, g, m, v);
+                const float pn = update<PRECISE, P_BF16 && !PRECISE>(r, p, g, m, v);
                 if (P_BF16) *(unsigned short*)(pp + e * 2) = __bfloat16_as_ushort(__float2bfloat16_rn(pn));
                 else *(float*)(pp + e * 4) = pn;
                 mp[e] = m;

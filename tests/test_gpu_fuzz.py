@@ -1,0 +1,51 @@
+"""Seeded random configurations (block size, tensor sizes and alignment, parameter / gradient / state types,
+hyper-parameters, gradient scale, number of steps) against the oracle. Every step is compared from identical
+inputs: after each comparison the oracle takes over the GPU's parameters (the state has to be identical
+anyway), so a one-ulp difference that the tolerance allows at one step cannot be magnified by a later step
+that shrinks the parameter."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_11919_b200 import workloads as W
+from test_gpu_parity import run_free
+
+pytestmark = pytest.mark.gpu
+
+
+def make_case(case: int, bf16_params=None):
+    rng = np.random.default_rng(1000 + case)
+    block = int(rng.choice([256, 512, 1024, 2048, 2048, 4096, 4096, 8192, 16384]))
+    nt = int(rng.integers(1, 120))
+    mult = int(rng.choice([block, 4, 8, 16, 2048]))
+    spec = W.ragged_spec(n_tensors=nt, max_numel=int(rng.choice([1 << 12, 1 << 15, 1 << 17, 1 << 19])), seed=case,
+                         multiple=mult)
+    bf16 = rng.uniform() < 0.5
+    spec.param_dtype = torch.bfloat16 if (bf16 if bf16_params is None else bf16_params) else torch.float32
+    spec.grad_dtype = torch.float32 if rng.uniform() < 0.25 else torch.bfloat16
+    spec.align_elems = int(rng.choice([1, 1, 2, 4, 8, 16]))
+    if rng.uniform() < 0.4:
+        spec.state_f32 = [bool(rng.uniform() < 0.5) for _ in spec.sizes]
+    spec.grad_std = float(10.0 ** rng.uniform(-6, 0))
+    spec.max_norm = float(rng.choice([0.5, 1.0, 1e-3, 100.0]))
+    hp = dict(lr=float(10.0 ** rng.uniform(-6, -3)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95])),
+              beta2=float(rng.choice([0.5, 0.95, 0.999, 0.9999])), eps=float(rng.choice([1e-8, 1e-6, 1e-10])),
+              weight_decay=float(rng.choice([0.0, 0.01, 0.1])))
+    steps = int(rng.integers(1, 5))
+    return spec, block, hp, steps
+
+
+@pytest.mark.parametrize("first", [0, 25, 50, 75])
+def test_random_configurations(first):
+    for case in range(first, first + 25):
+        spec, block, hp, steps = make_case(case)
+        run_free(spec, block, steps, hp_kw=hp, resync=True)
+
+
+@pytest.mark.parametrize("case", [2449, 2567])
+def test_parameter_cancelling_against_its_update(case):
+    # bf16 parameters, found by a longer run of the generator above: an element whose decayed parameter and
+    # update cancel to a few thousandths of either. Without the kernel's cancellation guard the approximate
+    # update's error (1e-7 of the update) is 2 to 3 bf16 ulps of that tiny result.
+    spec, block, hp, steps = make_case(case, bf16_params=True)
+    run_free(spec, block, steps, hp_kw=hp, resync=True)

@@ -24,8 +24,10 @@ def to_bf16_params(spec):
     return spec
 
 
-def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True):
-    """GPU and oracle run `steps` steps independently from the same start; returns per-step stats."""
+def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True, resync=False):
+    """GPU and oracle run `steps` steps independently from the same start; returns per-step stats.
+    resync: after every comparison the oracle takes over the GPU's parameters, so that each step is
+    compared from identical inputs (the state is compared for identity anyway)."""
     torch.cuda.set_device(0)
     buf = W.Buffers(spec, block, DEV)
     W.fill_params(buf)
@@ -61,9 +63,12 @@ def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True)
         assert int(opt.status.item()) == 0
         if check_every_step or k == steps:
             st = compare(buf, ots, slices)
-            st.norm_rel = abs(S_gpu - S) / S
+            st.norm_rel = abs(S_gpu - S) / S if S else 0.0
             st.check()
             out.append(st)
+        if resync:
+            for ot, (t_, b0, nb) in zip(ots, slices):
+                ot.param[:] = host_np(buf.view("param", t_))
     return out
 
 
