@@ -116,7 +116,9 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
  * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). The parameter
  * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-15 or, for bf16
- * parameters, a step size lr / (1 - beta1^t) above 1e-4, where it is IEEE-exact as well. */
+ * parameters, a step size lr / (1 - beta1^t) above 1e-4, where it is IEEE-exact as well; bf16 parameters that
+ * cancel against their update to below 2^-11 of themselves also take the exact formula, so that the rounded
+ * result stays within one bf16 ulp of the definition. */
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 
