@@ -33,7 +33,7 @@ UNIT = "params/s"
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch / parameters of that launch, block 2048;
 # profiles/step_kernel_small.md). Traffic grows in proportion to the parameters, so a full launch's
 # traffic is this figure times its parameters.
-STEP_TRAFFIC_BYTES_PER_PARAM = {"f32": 13.92, "bf16": 9.92}
+STEP_TRAFFIC_BYTES_PER_PARAM = {"f32": 13.95, "bf16": 9.91}
 
 
 def algorithmic_bytes_per_param(param_bytes: int, block: int):
