@@ -1,5 +1,5 @@
 """Seeded random configurations (block size, tensor sizes and alignment, parameter / gradient / state types,
-hyper-parameters, gradient scale, number of steps) against the oracle. Every step is compared from identical
+hyper-parameters, gradient scale, number of steps, chunking of the list) against the oracle. Every step is compared from identical
 inputs: after each comparison the oracle takes over the GPU's parameters (the state has to be identical
 anyway), so a one-ulp difference that the tolerance allows at one step cannot be magnified by a later step
 that shrinks the parameter."""
@@ -32,14 +32,19 @@ def make_case(case: int, bf16_params=None):
               beta2=float(rng.choice([0.5, 0.95, 0.999, 0.9999])), eps=float(rng.choice([1e-8, 1e-6, 1e-10])),
               weight_decay=float(rng.choice([0.0, 0.01, 0.1])))
     steps = int(rng.integers(1, 5))
-    return spec, block, hp, steps
+    chunks = None
+    if rng.uniform() < 0.3 and nt >= 4:          # the list updated in two to four calls under one norm
+        cuts = sorted(set(int(c) for c in rng.integers(1, nt, size=int(rng.integers(1, 4)))))
+        bounds = [0] + cuts + [nt]
+        chunks = [list(range(a, b)) for a, b in zip(bounds[:-1], bounds[1:])]
+    return spec, block, hp, steps, chunks
 
 
 @pytest.mark.parametrize("first", [0, 25, 50, 75])
 def test_random_configurations(first):
     for case in range(first, first + 25):
-        spec, block, hp, steps = make_case(case)
-        run_free(spec, block, steps, hp_kw=hp, resync=True)
+        spec, block, hp, steps, chunks = make_case(case)
+        run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
 
 
 @pytest.mark.parametrize("case", [2449, 2567])
@@ -47,5 +52,5 @@ def test_parameter_cancelling_against_its_update(case):
     # bf16 parameters, found by a longer run of the generator above: an element whose decayed parameter and
     # update cancel to a few thousandths of either. Without the kernel's cancellation guard the approximate
     # update's error (1e-7 of the update) is 2 to 3 bf16 ulps of that tiny result.
-    spec, block, hp, steps = make_case(case, bf16_params=True)
-    run_free(spec, block, steps, hp_kw=hp, resync=True)
+    spec, block, hp, steps, chunks = make_case(case, bf16_params=True)
+    run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
