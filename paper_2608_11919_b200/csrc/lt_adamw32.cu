@@ -10,6 +10,8 @@
 // approximate sqrt/reciprocal unless eps is tiny, as in the 8-bit kernel.
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "lt_common.cuh"
 
 namespace lt {
@@ -135,15 +137,16 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
 
 template <bool PRECISE, bool P_BF16>
 int launch(const StepParams& p, int sm_count, cudaStream_t s) {
-    static int grid_of_device[kMaxDevices] = {0};
+    static std::atomic<int> grid_of_device[kMaxDevices];   // racing host threads store the same value
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return LT_ERR_CUDA; }
-    int& full_grid = grid_of_device[dev];
+    int full_grid = grid_of_device[dev].load(std::memory_order_acquire);
     if (full_grid == 0) {
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adamw32_kernel<PRECISE, P_BF16>, kNT, 0) != cudaSuccess ||
             per_sm < 1) { cudaGetLastError(); return LT_ERR_CUDA; }
         full_grid = per_sm * sm_count;
+        grid_of_device[dev].store(full_grid, std::memory_order_release);
     }
     const int grid = p.total_blocks < full_grid ? p.total_blocks : full_grid;
     adamw32_kernel<PRECISE, P_BF16><<<grid, kNT, 0, s>>>(p);
