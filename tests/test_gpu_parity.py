@@ -263,6 +263,49 @@ def test_byte_zero_state_equals_value_zero_state():
         assert torch.equal(getattr(res[0], key), getattr(res[1], key)), key
 
 
+def test_two_host_threads_on_two_streams():
+    # two optimizers with their own buffers, scratch and streams, driven from two host threads at once
+    # (ctypes drops the GIL inside the library): each must end exactly where it ends when run alone
+    import threading
+    torch.cuda.set_device(0)
+    specs = [W.ragged_spec(n_tensors=200, max_numel=1 << 16, seed=51),
+             to_bf16_params(W.ragged_spec(n_tensors=150, max_numel=1 << 16, seed=52))]
+
+    def run(spec, block, stream, out, barrier=None):
+        torch.cuda.set_device(0)
+        with torch.cuda.stream(stream):
+            buf = W.Buffers(spec, block, DEV)
+            W.fill_params(buf)
+            opt = L.Hybrid8Optimizer(L.TensorList.from_buffers(buf), block, L.HParams(max_norm=0.5))
+            opt.init_state()
+            if barrier is not None:
+                barrier.wait()
+            for k in range(1, 9):
+                W.fill_grads(buf, k)
+                opt.step()
+            stream.synchronize()
+            out.append({k: getattr(buf, k).clone() for k in ("param", "m_code", "v_code", "m_absmax", "v_absmax")})
+
+    alone = []
+    for spec, block in zip(specs, (2048, 4096)):
+        res = []
+        run(spec, block, torch.cuda.Stream(), res)
+        alone.append(res[0])
+    together = [[], []]
+    barrier = threading.Barrier(2)
+    threads = [threading.Thread(target=run, args=(spec, block, torch.cuda.Stream(), together[i], barrier))
+               for i, (spec, block) in enumerate(zip(specs, (2048, 4096)))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+        assert not t.is_alive()
+    for a, b in zip(alone, together):
+        assert len(b) == 1
+        for k, v in a.items():
+            assert torch.equal(v, b[0][k]), k
+
+
 def test_resume_from_saved_state_is_bit_identical():
     torch.cuda.set_device(0)
     spec = W.ragged_spec(n_tensors=64, max_numel=1 << 15, seed=12)
