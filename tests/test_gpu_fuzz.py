@@ -13,7 +13,7 @@ from test_gpu_parity import run_free
 pytestmark = pytest.mark.gpu
 
 
-def make_case(case: int, bf16_params=None):
+def make_case(case: int, bf16_params=None, lr_max_exp: float = -3.0):
     rng = np.random.default_rng(1000 + case)
     block = int(rng.choice([256, 512, 1024, 2048, 2048, 4096, 4096, 8192, 16384]))
     nt = int(rng.integers(1, 120))
@@ -28,7 +28,7 @@ def make_case(case: int, bf16_params=None):
         spec.state_f32 = [bool(rng.uniform() < 0.5) for _ in spec.sizes]
     spec.grad_std = float(10.0 ** rng.uniform(-6, 0))
     spec.max_norm = float(rng.choice([0.5, 1.0, 1e-3, 100.0]))
-    hp = dict(lr=float(10.0 ** rng.uniform(-6, -3)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95])),
+    hp = dict(lr=float(10.0 ** rng.uniform(-6, lr_max_exp)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95])),
               beta2=float(rng.choice([0.5, 0.95, 0.999, 0.9999])), eps=float(rng.choice([1e-8, 1e-6, 1e-10])),
               weight_decay=float(rng.choice([0.0, 0.01, 0.1])))
     steps = int(rng.integers(1, 5))
@@ -54,3 +54,11 @@ def test_parameter_cancelling_against_its_update(case):
     # update's error (1e-7 of the update) is 2 to 3 bf16 ulps of that tiny result.
     spec, block, hp, steps, chunks = make_case(case, bf16_params=True)
     run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
+
+
+def test_bf16_parameters_at_large_learning_rates():
+    # learning rates up to 0.3: update and parameter are of one size, so they cancel often; every launch stays on
+    # the approximate path with its guard (there is no switch to the exact path by step size)
+    for case in range(20000, 20040):
+        spec, block, hp, steps, chunks = make_case(case, bf16_params=True, lr_max_exp=-0.5)
+        run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
