@@ -115,9 +115,10 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  * are skipped", training-configuration table); the caller clears d_status when it wants to.
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
  * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). The parameter
- * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-15, where it
- * is IEEE-exact as well; bf16 parameters that cancel against their update to below 2^-11 of themselves
- * also take the exact formula, so that the rounded result stays within one bf16 ulp of the definition. */
+ * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-15 or, for fp32
+ * parameters, a step size lr / (1 - beta1^t) above 5e-4, where it is IEEE-exact as well; bf16 parameters that
+ * cancel against their update to below 2^-11 of themselves also take the exact formula, so that the rounded
+ * result stays within one bf16 ulp of the definition. */
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 
@@ -152,7 +153,8 @@ typedef struct {
 int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, lt_stream stream);
 
 /* lt_hybrid8_step with the step count taken from the device: identical except that hp->step is ignored
- * and step_size / inv_sqrt_bc2 are read from *d_state by the kernels. */
+ * and step_size / inv_sqrt_bc2 are read from *d_state by the kernels. fp32 parameters take the exact
+ * parameter path when lr / (1 - beta1) > 5e-4 (the largest step size any count can give). */
 int lt_hybrid8_step_graph(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                           const lt_step_state* d_state, const double* d_sqnorm, int32_t* d_status,
                           lt_stream stream);

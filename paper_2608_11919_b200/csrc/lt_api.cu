@@ -334,7 +334,7 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     if (use_state) {
         if (!d_state) return LT_ERR_INVALID_ARG;
         if (!aligned(d_state, 8)) return LT_ERR_ALIGNMENT;
-        hp_local.step = 1;   // a valid count for the checks below; the kernels read the real scalars from *d_state
+        hp_local.step = 1;   // the largest step size any count can give (rule below); the kernels read the real scalars
     }
     const lt_hparams* hp = &hp_local;
     int rc = validate_tensors(tensors, n, NEED_GRAD | NEED_PARAM | NEED_STATE);
@@ -363,16 +363,19 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     P.s.clip_on = clip_on ? 1 : 0;
     // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps
     const bool precise_any = hp->eps < 1e-15f;
-    // (bf16 parameters need no rule of their own: where the approximate update's ~2^-21 relative error could show
-    // after rounding to bf16 -- parameter and update cancelling -- the kernels' cancellation guard takes the
-    // exact formula for that element, at any step size)
+    // Where parameter and update cancel, the approximate update's ~2^-21 relative error is large against the
+    // small result. bf16 launches carry a per-element guard for that (any step size). fp32 parameters are
+    // held to 1e-5 of max(|p|, 1e-3), which such an error can only exceed when the update itself exceeds
+    // 0.02, i.e. (|m'| / sqrt(v') stays below a few tens) at step sizes no sane AdamW run uses: those
+    // launches simply take the exact path.
+    const bool precise_f32 = precise_any || P.s.step_size > 5e-4f;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
     P.dev_scalars = use_state ? &d_state->step_size : nullptr;
     for (int st = LT_STATE_U8; st <= LT_STATE_F32; ++st) {
         for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype and one state kind per launch
             P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
-            P.s.precise_param = precise_any ? 1 : 0;
+            P.s.precise_param = (dt == LT_F32 ? precise_f32 : precise_any) ? 1 : 0;
             int32_t i = 0;
             while (i < n) {
                 pack_step(tensors, n, st == LT_STATE_F32 ? kAdamw32Item : block, &i, &P, true, dt, st);
