@@ -103,14 +103,23 @@ def compare(buf: W.Buffers, ots, slices, stats: Stats | None = None) -> Stats:
         n = ot.numel
         nbk = ot.m_absmax.size
         gp = host_np(buf.view("param", t)[e0:e0 + n])
+        # a NaN parameter (0/0 with eps = 0 on an element whose moments are zero) must be NaN on both sides;
+        # its bit pattern is nobody's business
         if ot.param.dtype == np.float32:
             ref = ot.param.astype(np.float64)
-            err = np.abs(gp.astype(np.float64) - ref) / np.maximum(np.abs(ref), PARAM_FLOOR / PARAM_RTOL)
+            got = gp.astype(np.float64)
+            same = (np.isnan(ref) & np.isnan(got)) | (got == ref)          # equal values include equal infinities
+            with np.errstate(invalid="ignore"):
+                err = np.abs(got - ref) / np.maximum(np.abs(ref), PARAM_FLOOR / PARAM_RTOL)
+            err = np.where(same, 0.0, np.where(np.isnan(err), np.inf, err))
             if n:
                 st.param_max_rel = max(st.param_max_rel, float(err.max()))
         else:
             if n:
-                st.param_max_ulp = max(st.param_max_ulp, int(np.abs(_bf16_ordinal(gp) - _bf16_ordinal(ot.param)).max()))
+                is_nan = lambda b: (b & 0x7FFF) > 0x7F80      # noqa: E731
+                d = np.abs(_bf16_ordinal(gp) - _bf16_ordinal(ot.param))
+                d = np.where(is_nan(gp) & is_nan(ot.param), 0, d)
+                st.param_max_ulp = max(st.param_max_ulp, int(d.max()))
         if ot.fp32_state:                 # plain fp32 moments: compared as values
             for key in ("m_code", "v_code"):
                 g = host_np(buf.view(key, t)[e0:e0 + n]).astype(np.float64)

@@ -13,7 +13,7 @@ from test_gpu_parity import run_free
 pytestmark = pytest.mark.gpu
 
 
-def make_case(case: int, bf16_params=None, lr_max_exp: float = -3.0):
+def make_case(case: int, bf16_params=None, lr_max_exp: float = -3.0, extreme: bool = False):
     rng = np.random.default_rng(1000 + case)
     block = int(rng.choice([256, 512, 1024, 2048, 2048, 4096, 4096, 8192, 16384]))
     nt = int(rng.integers(1, 120))
@@ -26,11 +26,19 @@ def make_case(case: int, bf16_params=None, lr_max_exp: float = -3.0):
     spec.align_elems = int(rng.choice([1, 1, 2, 4, 8, 16]))
     if rng.uniform() < 0.4:
         spec.state_f32 = [bool(rng.uniform() < 0.5) for _ in spec.sizes]
-    spec.grad_std = float(10.0 ** rng.uniform(-6, 0))
+    spec.grad_std = float(10.0 ** (rng.uniform(-12, 4) if extreme else rng.uniform(-6, 0)))
     spec.max_norm = float(rng.choice([0.5, 1.0, 1e-3, 100.0]))
-    hp = dict(lr=float(10.0 ** rng.uniform(-6, lr_max_exp)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95])),
-              beta2=float(rng.choice([0.5, 0.95, 0.999, 0.9999])), eps=float(rng.choice([1e-8, 1e-6, 1e-10])),
-              weight_decay=float(rng.choice([0.0, 0.01, 0.1])))
+    if extreme:
+        hp = dict(lr=float(10.0 ** rng.uniform(-6, lr_max_exp)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95, 0.999])),
+                  beta2=float(rng.choice([0.0, 0.5, 0.95, 0.999, 0.99999])),
+                  eps=float(rng.choice([0.0, 1e-12, 1e-8, 1e-6, 1e-3, 1.0])),
+                  weight_decay=float(rng.choice([0.0, 0.01, 0.1, 1.0, 10.0])))
+        if hp["eps"] == 0.0:
+            spec.zero_grad_frac = 0.0        # whole tensors of 0/0 are nobody's parity case (single elements stay)
+    else:
+        hp = dict(lr=float(10.0 ** rng.uniform(-6, lr_max_exp)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95])),
+                  beta2=float(rng.choice([0.5, 0.95, 0.999, 0.9999])), eps=float(rng.choice([1e-8, 1e-6, 1e-10])),
+                  weight_decay=float(rng.choice([0.0, 0.01, 0.1])))
     steps = int(rng.integers(1, 5))
     chunks = None
     if rng.uniform() < 0.3 and nt >= 4:          # the list updated in two to four calls under one norm
@@ -70,4 +78,12 @@ def test_fp32_parameters_at_large_learning_rates():
     # before that rule)
     for case in range(32361, 32480, 3):
         spec, block, hp, steps, chunks = make_case(case, bf16_params=False, lr_max_exp=-0.5)
+        run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
+
+
+def test_extreme_hyper_parameters_and_gradient_scales():
+    # gradient scales from 1e-12 to 1e4, eps from 0 to 1, weight decay up to 10, beta2 = 0: overflow to Inf and
+    # 0/0 do occur, and must occur on both sides alike (the comparison requires equal NaN-ness and equal infinities)
+    for case in range(40000, 40060):
+        spec, block, hp, steps, chunks = make_case(case, extreme=True)
         run_free(spec, block, steps, hp_kw=hp, chunks=chunks, resync=True)
