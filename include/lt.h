@@ -115,7 +115,7 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  * are skipped", training-configuration table); the caller clears d_status when it wants to.
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
  * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). The parameter
- * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-15 or, for fp32
+ * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-12 or, for fp32
  * parameters, a step size lr / (1 - beta1^t) above 5e-4, where it is IEEE-exact as well; bf16 parameters that
  * cancel against their update to below 2^-11 of themselves also take the exact formula, so that the rounded
  * result stays within one bf16 ulp of the definition. */

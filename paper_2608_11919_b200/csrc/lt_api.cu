@@ -362,7 +362,8 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     P.s.max_norm = hp->max_norm;
     P.s.clip_on = clip_on ? 1 : 0;
     // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps
-    const bool precise_any = hp->eps < 1e-15f;
+    // (sqrt of a subnormal v' is at most 1.1e-19: against eps >= 1e-12 its loss is below 1.1e-7 of the denominator)
+    const bool precise_any = hp->eps < 1e-12f;
     // Where parameter and update cancel, the approximate update's ~2^-21 relative error is large against the
     // small result. bf16 launches carry a per-element guard for that (any step size). fp32 parameters are
     // held to 1e-5 of max(|p|, 1e-3), which such an error can only exceed when the update itself exceeds
