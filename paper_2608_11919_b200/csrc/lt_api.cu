@@ -359,6 +359,7 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     P.s.inv_sqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
     P.s.decay = (float)(1.0 - (double)hp->lr * (double)hp->weight_decay);
     P.s.eps = hp->eps;
+    P.s.one = 1.0f;
     P.s.max_norm = hp->max_norm;
     P.s.clip_on = clip_on ? 1 : 0;
     // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps

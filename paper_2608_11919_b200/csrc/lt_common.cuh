@@ -34,6 +34,7 @@ struct StepDesc {               // 64 bytes
 
 struct StepScalars {
     float beta1, beta2, omb1, omb2, step_size, inv_sqrt_bc2, decay, eps, max_norm;
+    float one;                  // 1.0f, a run-time value on purpose (lt_step.cu, add2_rt)
     int32_t clip_on;
     int32_t precise_param;      // 1: IEEE sqrt and divide in the parameter update (tiny eps)
 };
