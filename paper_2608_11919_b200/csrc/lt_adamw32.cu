@@ -13,6 +13,7 @@
 #include <atomic>
 
 #include "lt_common.cuh"
+#include "lt_update.cuh"
 
 namespace lt {
 
@@ -21,49 +22,33 @@ namespace {
 constexpr int kNT = 256;
 constexpr int kK = kAdamw32Item / (4 * kNT);
 
-struct Regs { float c, beta1, beta2, omb1, omb2, step_size, isb2, decay, eps; };
-
-__device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
-__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
-
-// The parameter update exactly as defined (IEEE sqrt and divide, one rounding per operation).
-__device__ __forceinline__ float param_exact(const Regs& r, float p, float m, float v) {
-    const float den = __fadd_rn(__fmul_rn(__fsqrt_rn(v), r.isb2), r.eps);
-    return __fsub_rn(__fmul_rn(p, r.decay), __fmul_rn(r.step_size, __fdiv_rn(m, den)));
-}
-
-// One element. GUARD (bf16 parameters on the approximate path): when p * decay and the update cancel to below
-// 2^-11 of p * decay, the approximate update's error (~2^-21 of the update) would be worth more than one bf16
-// ulp of the tiny result; such elements (about 2 in 10^7) take the exact formula. Same rule as the step kernel.
+// Two elements: moments in place, new parameters returned. GUARD (bf16 parameters on the approximate path):
+// an element whose result cancels below 2^-11 of p * decay takes the exact formula (cancel_risk, lt_update.cuh).
 template <bool PRECISE, bool GUARD>
-__device__ __forceinline__ float update(const Regs& r, float p, float g, float& m, float& v) {
-    const float gc = __fmul_rn(g, r.c);
-    m = __fadd_rn(__fmul_rn(r.beta1, m), __fmul_rn(r.omb1, gc));
-    v = __fadd_rn(__fmul_rn(r.beta2, v), __fmul_rn(r.omb2, __fmul_rn(gc, gc)));
-    if (PRECISE) return param_exact(r, p, m, v);
-    const float den = __fmaf_rn(sqrt_approx(v), r.isb2, r.eps);
-    const float pd = __fmul_rn(p, r.decay);                                        // rounded first, as defined
-    const float pn = __fmaf_rn(-r.step_size, __fmul_rn(m, rcp_approx(den)), pd);
-    if (GUARD && __fmaf_rn(fabsf(pn), 2048.0f, -fabsf(pd)) < 0.0f) return param_exact(r, p, m, v);
+__device__ __forceinline__ float2 update2(const StepRegs& r, float2 p, float2 g, float2& m, float2& v) {
+    float2 pd;
+    moments_pair(r, g, m, v, m, v);
+    float2 pn = param_pair<PRECISE>(r, p, m, v, pd);
+    if (GUARD && fminf(cancel_risk(pn.x, pd.x), cancel_risk(pn.y, pd.y)) < 0.0f) {
+        pn.x = param_exact(r, p.x, m.x, v.x);
+        pn.y = param_exact(r, p.y, m.y, v.y);
+    }
+    return pn;
+}
+template <bool PRECISE, bool GUARD>
+__device__ __forceinline__ float update(const StepRegs& r, float p, float g, float& m, float& v) {
+    float pd;
+    moments_one(r, g, m, v, m, v);
+    const float pn = param_one<PRECISE>(r, p, m, v, pd);
+    if (GUARD && cancel_risk(pn, pd) < 0.0f) return param_exact(r, p, m, v);
     return pn;
 }
 
 template <bool PRECISE, bool P_BF16>
 __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ StepParams P) {
     const int tid = threadIdx.x;
-    Regs r;
-    r.c = 1.0f;
-    if (P.sqnorm != nullptr) {
-        const double S = *P.sqnorm;
-        if (!isfinite(S)) {
-            if (blockIdx.x == 0 && tid == 0 && P.status != nullptr) atomicOr(P.status, 1);
-            return;
-        }
-        if (P.s.clip_on) r.c = (float)fmin(1.0, (double)P.s.max_norm / (sqrt(S) + 1e-6));
-    }
-    r.beta1 = P.s.beta1; r.beta2 = P.s.beta2; r.omb1 = P.s.omb1; r.omb2 = P.s.omb2;
-    r.step_size = P.s.step_size; r.isb2 = P.s.inv_sqrt_bc2; r.decay = P.s.decay; r.eps = P.s.eps;
-    if (P.dev_scalars != nullptr) { r.step_size = P.dev_scalars[0]; r.isb2 = P.dev_scalars[1]; }
+    StepRegs r;
+    if (!load_step_regs(P, r)) return;
 
     int t = 0, begin = 0;
     for (int w = blockIdx.x; w < P.total_blocks; w += gridDim.x) {
@@ -101,10 +86,13 @@ __global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ St
                 }
                 g[0] = __uint_as_float(gr[k].x << 16); g[1] = __uint_as_float(gr[k].x & 0xffff0000u);
                 g[2] = __uint_as_float(gr[k].y << 16); g[3] = __uint_as_float(gr[k].y & 0xffff0000u);
-                pn[0] = update<PRECISE, P_BF16 && !PRECISE>(r, p[0], g[0], mr[k].x, vr[k].x);
-                pn[1] = update<PRECISE, P_BF16 && !PRECISE>(r, p[1], g[1], mr[k].y, vr[k].y);
-                pn[2] = update<PRECISE, P_BF16 && !PRECISE>(r, p[2], g[2], mr[k].z, vr[k].z);
-                pn[3] = update<PRECISE, P_BF16 && !PRECISE>(r, p[3], g[3], mr[k].w, vr[k].w);
+                float2 m01 = make_float2(mr[k].x, mr[k].y), m23 = make_float2(mr[k].z, mr[k].w);
+                float2 v01 = make_float2(vr[k].x, vr[k].y), v23 = make_float2(vr[k].z, vr[k].w);
+                const float2 n01 = update2<PRECISE, P_BF16 && !PRECISE>(r, make_float2(p[0], p[1]), make_float2(g[0], g[1]), m01, v01);
+                const float2 n23 = update2<PRECISE, P_BF16 && !PRECISE>(r, make_float2(p[2], p[3]), make_float2(g[2], g[3]), m23, v23);
+                pn[0] = n01.x; pn[1] = n01.y; pn[2] = n23.x; pn[3] = n23.y;
+                mr[k] = make_float4(m01.x, m01.y, m23.x, m23.y);
+                vr[k] = make_float4(v01.x, v01.y, v23.x, v23.y);
                 if (P_BF16) {
                     const __nv_bfloat162 lo = __floats2bfloat162_rn(pn[0], pn[1]);
                     const __nv_bfloat162 hi = __floats2bfloat162_rn(pn[2], pn[3]);

@@ -362,22 +362,20 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     P.s.one = 1.0f;
     P.s.max_norm = hp->max_norm;
     P.s.clip_on = clip_on ? 1 : 0;
-    // the fast parameter update flushes subnormal v' to zero, harmless only against a sane eps
-    // (sqrt of a subnormal v' is at most 1.1e-19: against eps >= 1e-12 its loss is below 1.1e-7 of the denominator)
-    const bool precise_any = hp->eps < 1e-12f;
-    // Where parameter and update cancel, the approximate update's ~2^-21 relative error is large against the
-    // small result. bf16 launches carry a per-element guard for that (any step size). fp32 parameters are
-    // held to 1e-5 of max(|p|, 1e-3), which such an error can only exceed when the update itself exceeds
-    // 0.02, i.e. (|m'| / sqrt(v') stays below a few tens) at step sizes no sane AdamW run uses: those
-    // launches simply take the exact path.
-    const bool precise_f32 = precise_any || P.s.step_size > 5e-4f;
+    // The approximate parameter update (hardware sqrt and reciprocal approximations) is within
+    // 6.6e-7 |update| + 1.2e-7 |p'| of the defined one (derivation in lt_update.cuh): inside 1e-5 of
+    // max(|p'|, |update|) for fp32 parameters at any step size, and inside one bf16 ulp under the kernels'
+    // cancellation guard. One case is outside that derivation: the fast path flushes a subnormal v' to zero,
+    // which is harmless only against a sane eps (sqrt of a subnormal is at most 1.1e-19: against
+    // eps >= 1e-12 its loss is below 1.1e-7 of the denominator). Smaller eps takes the exact path.
+    const bool precise = hp->eps < 1e-12f;
     P.sqnorm = d_sqnorm;
     P.status = d_status;
     P.dev_scalars = use_state ? &d_state->step_size : nullptr;
     for (int st = LT_STATE_U8; st <= LT_STATE_F32; ++st) {
         for (int dt = LT_F32; dt <= LT_BF16; ++dt) {   // one parameter dtype and one state kind per launch
             P.param_bf16 = (dt == LT_BF16) ? 1 : 0;
-            P.s.precise_param = (dt == LT_F32 ? precise_f32 : precise_any) ? 1 : 0;
+            P.s.precise_param = precise ? 1 : 0;
             int32_t i = 0;
             while (i < n) {
                 pack_step(tensors, n, st == LT_STATE_F32 ? kAdamw32Item : block, &i, &P, true, dt, st);

@@ -12,7 +12,7 @@ import torch
 import oracle as O
 import paper_2608_11919_b200 as L
 from paper_2608_11919_b200 import workloads as W
-from parity_util import (NORM_RTOL, Stats, compare, host_np, oracle_sqnorm_of_buffers, oracle_tensors,
+from parity_util import (NORM_RTOL, Stats, adopt_gpu_params, compare, host_np, oracle_sqnorm_of_buffers, oracle_step, oracle_tensors,
                          parallel_oracle_step, refresh_grads)
 
 pytestmark = pytest.mark.gpu
@@ -67,8 +67,7 @@ def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True,
             st.check()
             out.append(st)
         if resync:
-            for ot, (t_, b0, nb) in zip(ots, slices):
-                ot.param[:] = host_np(buf.view("param", t_))
+            adopt_gpu_params(ots, buf, slices)
     return out
 
 
@@ -92,7 +91,7 @@ def test_forty_free_running_steps_do_not_drift():
         spec.step_scale = {2: 1e3, 7: 1e-2, 13: 50.0}
         stats = run_free(spec, 2048, 40, check_every_step=False)
         assert stats[-1].code_mismatch == 0 and stats[-1].scale_max_rel == 0.0
-        assert stats[-1].param_max_rel <= 5e-7 and stats[-1].param_max_ulp <= 1, stats[-1]
+        assert stats[-1].param_max_rel <= 1e-6 and stats[-1].param_max_ulp <= 1, stats[-1]   # the one-FMA form: 2.7e-6
 
 
 def test_tiny_unclipped_variant():
@@ -113,7 +112,7 @@ def test_tiny_clipping_disabled_null_norm():
     hp = L.HParams(max_norm=0.0)
     L.lt_hybrid8_step(tl, 2048, hp, None, None)
     torch.cuda.synchronize()
-    O.hybrid8_step(ots, 2048, O.HParams(max_norm=0.0), 1.0)
+    oracle_step(ots, 2048, O.HParams(max_norm=0.0), 1.0)
     compare(buf, ots, slices).check()
 
 
@@ -413,7 +412,7 @@ def test_late_step_count_and_infinite_max_norm():
         L.lt_grad_sqnorm_multi(tl, sq, ws)
         L.lt_hybrid8_step(tl, 4096, L.HParams(max_norm=float("inf"), step=t), sq, None)
         torch.cuda.synchronize()
-        O.hybrid8_step(ots, 4096, O.HParams(max_norm=float("inf"), step=t), O.sqnorm(ots))
+        oracle_step(ots, 4096, O.HParams(max_norm=float("inf"), step=t), O.sqnorm(ots))
         compare(buf, ots, slices).check()
 
 
