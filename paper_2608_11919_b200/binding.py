@@ -122,6 +122,20 @@ class TensorList:
         return cls(*[[buf.view(k, t) for t in idx]
                      for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax")])
 
+    @classmethod
+    def from_buffer_pieces(cls, buf, pieces) -> "TensorList":
+        """Descriptors over block-aligned pieces (tensor index, first block, number of blocks) of the tensors
+        of a `workloads.Buffers`, as `sharding.partition_blocks` hands them out."""
+        cols = [[] for _ in range(6)]
+        for t, b0, nb in pieces:
+            size = buf.spec.sizes[t]
+            e0, e1 = b0 * buf.block, min(size, (b0 + nb) * buf.block)
+            for c, k in zip(cols, ("param", "grad", "m_code", "v_code")):
+                c.append(buf.view(k, t)[e0:e1])
+            for c, k in zip(cols[4:], ("m_absmax", "v_absmax")):
+                c.append(buf.view(k, t)[b0:b0 + nb])
+        return cls(*cols)
+
     def slice(self, start: int, stop: int) -> "TensorList":
         return TensorList(*[x[start:stop] for x in self._keep])
 

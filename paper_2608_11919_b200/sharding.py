@@ -41,6 +41,31 @@ def partition_contiguous(sizes: Sequence[int], world: int) -> List[range]:
     return [range(cuts[r], cuts[r + 1]) for r in range(world)]
 
 
+def partition_blocks(sizes: Sequence[int], block: int, world: int) -> List[List[tuple]]:
+    """Balanced partition by QUANTIZATION BLOCKS rather than whole tensors: the list is read as one sequence
+    of blocks (tensor after tensor) and cut into `world` consecutive runs whose block counts differ by at most
+    one. Returns, per rank, pieces (tensor index, first block, number of blocks) in list order; a tensor that
+    straddles a cut is split at a block boundary, which changes nothing in the result because blocks are
+    independent once the global norm is known. This removes the imbalance a large embedding causes when whole
+    tensors are the unit (a tied 3B embedding is 10 % of the model)."""
+    assert world >= 1 and block >= 1
+    nbs = [(int(x) + block - 1) // block for x in sizes]
+    total = sum(nbs)
+    out: List[List[tuple]] = [[] for _ in range(world)]
+    t, used = 0, 0                       # next tensor, blocks of it already handed out
+    for r in range(world):
+        want = total * (r + 1) // world - total * r // world
+        while want > 0 and t < len(nbs):
+            take = min(want, nbs[t] - used)
+            if take > 0:
+                out[r].append((t, used, take))
+                used += take
+                want -= take
+            if used == nbs[t]:
+                t, used = t + 1, 0
+    return out
+
+
 def allgather_params(param_flat: torch.Tensor, bounds: Sequence[Sequence[int]], group=None) -> None:
     """For replicated parameters: after the step every rank has updated only the slice it owns;
     `bounds[r] = (begin, end)` is rank r's element range of `param_flat`. Each slice is broadcast from
@@ -71,12 +96,18 @@ def allreduce_sqnorm(sqnorm: torch.Tensor, group=None) -> None:
 
 
 class ShardedHybrid8:
-    """One rank's optimizer over the tensors it owns: norm (local) -> all-reduce -> step (local)."""
+    """One rank's optimizer over the tensors it owns: norm (local) -> all-reduce -> step (local).
+
+    `optimizer` is a Hybrid8Optimizer over this rank's tensors only. The step is split in its two phases
+    so that a caller without a process group (several shards driven by one process, as in the one-GPU
+    tests) can put its own reduction between them: norm_phase() of every shard, then reduce, then
+    update_phase() of every shard."""
 
     def __init__(self, optimizer, group=None):
         self.opt, self.group = optimizer, group
 
-    def step(self) -> None:
+    def norm_phase(self) -> None:
+        """S1 over the owned tensors: opt.sqnorm = this rank's partial sum of squares."""
         from . import binding as B
         o = self.opt
         o.t += 1
@@ -84,6 +115,16 @@ class ShardedHybrid8:
         o.sqnorm.zero_()
         for ch in o.chunks:
             B.lt_grad_sqnorm_multi(ch, o.sqnorm, o.workspace)
-        allreduce_sqnorm(o.sqnorm, self.group)
+
+    def update_phase(self) -> None:
+        """S2..S5 over the owned tensors; opt.sqnorm must hold the global sum by now."""
+        from . import binding as B
+        o = self.opt
+        B.lt_skip_count_update(o.sqnorm, o.skip_count)
         for ch in o.chunks:
             B.lt_hybrid8_step(ch, o.block, o.hp, o.sqnorm, o.status)
+
+    def step(self) -> None:
+        self.norm_phase()
+        allreduce_sqnorm(self.opt.sqnorm, self.group)
+        self.update_phase()

@@ -27,7 +27,7 @@ from __future__ import annotations
 
 import math
 from dataclasses import dataclass, field
-from typing import List, Optional
+from typing import List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -146,6 +146,17 @@ def small_bf16_spec() -> Spec:
 
 SPECS = {"7b_hybrid": lambda: hybrid_split(qwen7b_spec()), "small_hybrid": lambda: hybrid_split(small_spec()),
          "small": small_spec, "small_bf16": small_bf16_spec, "tiny": tiny_spec, "ragged": ragged_spec, "3b": qwen3b_spec, "7b": qwen7b_spec, "27b": dense27b_spec}
+
+
+def subset_spec(spec: Spec, indices: Sequence[int], suffix: str = "") -> Spec:
+    """The same workload restricted to the tensors `indices` (one rank's shard of the list). Layer indices
+    are kept, so layer grouping and per-layer gradient scales stay those of the full list."""
+    import dataclasses
+    idx = list(indices)
+    return dataclasses.replace(
+        spec, name=spec.name + suffix, names=[spec.names[i] for i in idx], sizes=[spec.sizes[i] for i in idx],
+        layer_of=[spec.layer_of[i] for i in idx], step_scale=dict(spec.step_scale),
+        state_f32=None if spec.state_f32 is None else [spec.state_f32[i] for i in idx])
 
 
 def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:

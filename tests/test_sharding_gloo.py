@@ -28,6 +28,22 @@ def test_partition_is_balanced_and_complete():
     assert max(loads) / (sum(loads) / 8) < 1.26                     # the tied embedding is 10 % of the model
 
 
+def test_block_partition_is_balanced_to_one_block():
+    for spec in (W.ragged_spec(n_tensors=300, max_numel=1 << 16, seed=2), W.qwen3b_spec(), W.dense27b_spec()):
+        nbs = [(s + BLOCK - 1) // BLOCK for s in spec.sizes]
+        for world in (1, 2, 3, 8):
+            parts = S.partition_blocks(spec.sizes, BLOCK, world)
+            flat = [x for p in parts for x in p]
+            covered = {}
+            for t, b0, nb in flat:                                  # every block exactly once, in list order
+                assert nb > 0 and b0 == covered.get(t, 0)
+                covered[t] = b0 + nb
+            assert covered == {t: n for t, n in enumerate(nbs) if n}
+            assert [x[0] for x in flat] == sorted(x[0] for x in flat)
+            loads = [sum(nb for _, _, nb in p) for p in parts]
+            assert max(loads) - min(loads) <= 1
+
+
 def _make(spec, step):
     buf = W.Buffers(spec, BLOCK, "cpu")
     W.fill_params(buf)
