@@ -309,7 +309,41 @@ def time_e2e(name, block, steps, warmup):
     return out
 
 
-def time_host_resident(name, block, steps):
+def link_probe(device, n_bytes: int = 1 << 28, reps: int = 6):
+    """Host link rates as this machine delivers them: pinned host <-> device copies of 256 MiB, one direction alone
+    and both directions at once (GB/s per direction)."""
+    import torch
+    h_in, h_out = torch.empty(n_bytes, dtype=torch.uint8).pin_memory(), torch.empty(n_bytes, dtype=torch.uint8).pin_memory()
+    d_in, d_out = torch.empty(n_bytes, dtype=torch.uint8, device=device), torch.empty(n_bytes, dtype=torch.uint8, device=device)
+    s_in, s_out = torch.cuda.Stream(device), torch.cuda.Stream(device)
+
+    def run(h2d, d2h):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        torch.cuda.synchronize()
+        for k in range(reps + 1):
+            if h2d:
+                with torch.cuda.stream(s_in):
+                    if k == 1:
+                        ev[0].record()
+                    d_in.copy_(h_in, non_blocking=True)
+            if d2h:
+                with torch.cuda.stream(s_out):
+                    if k == 1:
+                        ev[2].record()
+                    h_out.copy_(d_out, non_blocking=True)
+        if h2d:
+            ev[1].record(s_in)
+        if d2h:
+            ev[3].record(s_out)
+        torch.cuda.synchronize()
+        return (reps * n_bytes / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9 if h2d else None,
+                reps * n_bytes / (ev[2].elapsed_time(ev[3]) * 1e-3) / 1e9 if d2h else None)
+
+    return {"h2d_alone_gbs": run(True, False)[0], "d2h_alone_gbs": run(False, True)[1],
+            "h2d_with_d2h_gbs": run(True, True)[0], "d2h_with_h2d_gbs": run(True, True)[1]}
+
+
+def time_host_resident(name, block, steps, link=None):
     """The paper's own layout: parameters, gradients and state in pinned HOST memory, streamed through
     the kernels in layer-group chunks (paper_2608_11919_b200/host_resident.py); everything crosses the host
     link every step, in both directions."""
@@ -341,6 +375,13 @@ def time_host_resident(name, block, steps):
            "h2d_gbs": opt.h2d_bytes / (ms * 1e-3) / 1e9, "status": float(opt.result[1]),
            "what": "parameters, gradients and 8-bit state resident in pinned host memory; all of it copied in and the "
                    "updated parameters and state copied out every step, overlapped with the kernels"}
+    if link:
+        # the least time the link allows for these bytes: the return traffic overlaps as much inbound traffic
+        # at the both-directions rate, the rest of the inbound traffic runs alone
+        both = min(link["h2d_with_d2h_gbs"], link["d2h_with_h2d_gbs"])
+        floor = (opt.d2h_bytes / both + max(opt.h2d_bytes - opt.d2h_bytes, 0) / link["h2d_alone_gbs"]) / 1e9 * 1e3
+        out["link_floor_ms"] = floor
+        out["frac_of_link_floor"] = floor / ms
     del opt, host
     torch.cuda.empty_cache()
     return out
@@ -504,10 +545,10 @@ def main():
             e2e["d2h_bytes_per_step"] *= world
     host_state = None
     if not args.no_e2e and not dist_on and args.host_resident != "none":
-        host_state = {}
+        host_state = {"link": link_probe(torch.device("cuda", local))}
         for hw in [w.strip() for w in args.host_resident.split(",") if w.strip()]:
             try:
-                host_state[hw] = time_host_resident(hw, args.block, 3)
+                host_state[hw] = time_host_resident(hw, args.block, 3, host_state["link"])
             except (RuntimeError, MemoryError) as e:  # e.g. the host refuses to pin that much memory
                 host_state[hw] = {"workload": hw, "skipped": str(e)[:120]}
     cpu = cpu_all = None

@@ -1,6 +1,6 @@
 /* lt.h -- C ABI of the fused global-norm clip + block-wise 8-bit AdamW optimizer step (sm_100a).
  *
- * The operator is the optimizer-side component of the paper's Sec. 3.5 ("Hybrid 8-bit operator"):
+ * The operator is the optimizer-side component the paper calls the hybrid 8-bit operator (Sec. 3.5):
  * Adam moments held as 8-bit codes with block-wise scales, updated by an AdamW step, coupled with a
  * fast global-norm gradient clip. Here every step of it runs on the GPU, on the caller's stream.
  *
@@ -79,8 +79,8 @@ int lt_hybrid8_state_bytes(int64_t numel, int32_t block, int64_t* code_bytes, in
 
 /* Copies the 256-entry code map (signed: first moment, unsigned: second moment) to host memory.
  * Decade e = 0..6 with scale 10^(e-6) holds 2^e (signed) or 2^(e+1) (unsigned) cell mid-points of a
- * uniform grid on [0.1, 1]; plus 0.0 and +1.0 (the paper names only a "CPU 8-bit AdamW format", Sec.
- * 3.5; this map is this library's reading of it). */
+ * uniform grid on [0.1, 1]; plus 0.0 and +1.0 (the paper gives the format a name only -- an 8-bit AdamW
+ * format held in CPU memory, Sec. 3.5 --; this map is this library's reading of it). */
 int lt_hybrid8_code_table(int32_t is_signed, float* out256);
 
 /* Size in bytes of the device scratch lt_grad_sqnorm_multi needs (a constant, a few KB). The scratch
@@ -89,19 +89,23 @@ int lt_hybrid8_code_table(int32_t is_signed, float* out256);
 int64_t lt_workspace_bytes(void);
 
 /* S0 -- puts the 8-bit state of every tensor to value zero (m_code 127, v_code 0, scales 0).
- * Uses m_code, v_code, m_absmax, v_absmax, numel. (Sec. 3.5: moments "in CPU 8-bit AdamW format".) */
+ * Uses m_code, v_code, m_absmax, v_absmax, numel. (Sec. 3.5: the moments of the 8-bit slice are held in an
+ * 8-bit AdamW format.) */
 int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt_stream stream);
 
-/* S1 -- multi-tensor squared L2 norm (Sec. 3.5: the clip "computes per-tensor norms ... aggregates
- * the global norm"). ADDS sum_t sum_i grad[t][i]^2 to *d_sqnorm (device double). The caller zeroes
+/* S1 -- multi-tensor squared L2 norm (Sec. 3.5: the clip takes a norm per tensor and combines them into
+ * one global norm). ADDS sum_t sum_i grad[t][i]^2 to *d_sqnorm (device double). The caller zeroes
  * *d_sqnorm before the first chunk of an optimizer step and may call this once per chunk of the
- * tensor list. Uses grad, grad_dtype, numel. Accumulation is fp64 over exact fp32 squares; the
- * result is bit-reproducible for a given tensor list on a given device. */
+ * tensor list. Uses grad, grad_dtype, numel. Accumulation is fp64 over exact squares; the
+ * result is bit-reproducible for a given tensor list on a given device.
+ * The launch finishes with a plain read-add-write of *d_sqnorm by one thread: calls that accumulate into
+ * the same scalar must be ordered on the GPU (one stream, or events between streams). Two calls that may
+ * overlap need a scalar each (and a scratch buffer each); add the scalars afterwards. */
 int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
                          void* d_workspace, int64_t workspace_bytes, lt_stream stream);
 
-/* S2..S5 -- the fused step (Sec. 3.5: dequantize, "8-bit state updates", requantize with
- * "block-wise scale handling", under the clip's single scale). Reads S = *d_sqnorm, the squared norm
+/* S2..S5 -- the fused step (Sec. 3.5: dequantize the 8-bit moments, update them, requantize them with
+ * fresh per-block scales, all under the clip's single scale). Reads S = *d_sqnorm, the squared norm
  * over ALL gradients of this optimizer step (the tensor list may be one chunk of them):
  *     c   = min(1, max_norm / (sqrt(S) + 1e-6))                       (1 if clipping is disabled)
  *     g   = c * grad;   m = QS[m_code] * m_absmax[b];   v = QU[v_code] * v_absmax[b]
@@ -111,19 +115,27 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
  *     v'/v_absmax (ties to the lower index; an all-zero block gets zero codes and scale 0).
  * Tensors with state_dtype LT_STATE_F32 get the same update with m, v read and written as fp32 (no
  * tables, no block scales); both kinds may be mixed in one list and share the clip factor.
- * If S is NaN or Inf nothing is written except bit 0 of *d_status (the paper's "non-finite gradients
- * are skipped", training-configuration table); the caller clears d_status when it wants to.
+ * If S is NaN or Inf nothing is written except bit 0 of *d_status (the skip-on-non-finite rule of the
+ * paper's training-configuration table, safety-checks row); the caller clears d_status when it wants to.
  * d_sqnorm may be NULL only when clipping is disabled (no skip detection then). d_status may be NULL.
- * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add). The parameter
- * update uses approximate sqrt/reciprocal (a few fp32 ulp of the update), except with eps < 1e-12 or, for fp32
- * parameters, a step size lr / (1 - beta1^t) above 5e-4, where it is IEEE-exact as well; bf16 parameters that
- * cancel against their update to below 2^-11 of themselves also take the exact formula, so that the rounded
- * result stays within one bf16 ulp of the definition. */
+ * Status word: bit 0 (value 1) = this step was skipped because S is not finite. Bit 1 (value 2) = the
+ * kernel found its shared-memory window laid out differently from what it was built for and did nothing
+ * (a build or driver inconsistency, never expected; reported instead of risking a bad access). Bits are
+ * only ever set, by atomic OR.
+ * Moment arithmetic is IEEE fp32 with one rounding per operation (no fused multiply-add), so the stored
+ * state is that of a plain evaluation of the formulas above. The parameter update uses the hardware's
+ * approximate sqrt and reciprocal; its distance from the IEEE evaluation of the formula is bounded by
+ *     6.6e-7 |update| + 1.2e-7 |p_new|      (update = the term subtracted from p (1 - lr wd)),
+ * at any step size: within 1e-5 of max(|p_new|, |update|) for fp32 parameters. bf16 parameters whose result
+ * cancels to below 2^-11 of p (1 - lr wd) take the IEEE formula instead, which keeps every rounded result
+ * within one bf16 ulp (elements that are not flagged have |update| <= 2049 |p_new|, and the bound above is
+ * then below half a bf16 ulp). With eps < 1e-12 the whole launch takes the IEEE formula (the approximate
+ * sqrt flushes subnormal v'). */
 int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                     const double* d_sqnorm, int32_t* d_status, lt_stream stream);
 
-/* Per-tensor squared L2 norms, for logging (Sec. 3.5: the clip "computes per-tensor norms" before it
- * aggregates them). ADDS sum_i grad[t][i]^2 to d_out[t] for every tensor t of the list (device doubles,
+/* Per-tensor squared L2 norms, for logging (Sec. 3.5: the clip's first stage is a norm per tensor).
+ * ADDS sum_i grad[t][i]^2 to d_out[t] for every tensor t of the list (device doubles,
  * one per list entry, zeroed by the caller; entries of empty tensors are left alone). Uses grad,
  * grad_dtype, numel. Each addend is an exact fp64 square; per-CTA partial sums reach d_out[t] through
  * fp64 atomic adds, so the last bits may differ from run to run -- use lt_grad_sqnorm_multi for the norm
@@ -131,8 +143,8 @@ int lt_hybrid8_step(const lt_tensor* tensors, int32_t n, int32_t block, const lt
 int lt_grad_sqnorm_per_tensor(const lt_tensor* tensors, int32_t n, double* d_out, lt_stream stream);
 
 /* Skip bookkeeping, once per optimizer step, after the step's norm is complete (training-configuration
- * table: "Non-finite gradients are skipped; training aborts after three consecutive non-finite-gradient
- * events"). Reads S = *d_sqnorm and updates the device word *d_skip_count: S finite -> 0, S NaN/Inf ->
+ * table, safety-checks row: a step with non-finite gradients is skipped, and three such steps in a row end
+ * the run). Reads S = *d_sqnorm and updates the device word *d_skip_count: S finite -> 0, S NaN/Inf ->
  * previous value + 1. The caller reads it when it likes and applies its abort policy; nothing here
  * aborts. One thread of device work. */
 int lt_skip_count_update(const double* d_sqnorm, int32_t* d_skip_count, lt_stream stream);
@@ -149,12 +161,13 @@ typedef struct {
 
 /* One thread of device work: d_state->step += 1, then step_size and inv_sqrt_bc2 for the new count from
  * hp->lr, hp->beta1, hp->beta2 (formed in fp64, rounded once to fp32, like the host path; the device's
- * fp64 pow may differ from the host's in the last bit, which can move step_size by one fp32 ulp). */
-int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, lt_stream stream);
+ * fp64 pow may differ from the host's in the last bit, which can move step_size by one fp32 ulp).
+ * d_sqnorm (device, may be NULL): when given and *d_sqnorm is NaN or Inf, nothing changes -- the step that
+ * follows will be skipped, and a skipped step must not count towards the bias corrections. */
+int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, const double* d_sqnorm, lt_stream stream);
 
 /* lt_hybrid8_step with the step count taken from the device: identical except that hp->step is ignored
- * and step_size / inv_sqrt_bc2 are read from *d_state by the kernels. fp32 parameters take the exact
- * parameter path when lr / (1 - beta1) > 5e-4 (the largest step size any count can give). */
+ * and step_size / inv_sqrt_bc2 are read from *d_state by the kernels. */
 int lt_hybrid8_step_graph(const lt_tensor* tensors, int32_t n, int32_t block, const lt_hparams* hp,
                           const lt_step_state* d_state, const double* d_sqnorm, int32_t* d_status,
                           lt_stream stream);

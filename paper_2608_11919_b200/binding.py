@@ -55,7 +55,7 @@ def _load():
     L.lt_grad_sqnorm_multi_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.lt_grad_sqnorm_per_tensor.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.lt_skip_count_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
-    L.lt_step_state_advance.argtypes = [C.c_void_p, C.POINTER(_LtHParams), C.c_void_p]
+    L.lt_step_state_advance.argtypes = [C.c_void_p, C.POINTER(_LtHParams), C.c_void_p, C.c_void_p]
     L.lt_hybrid8_step_graph.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_LtHParams), C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.c_void_p]
     return L
@@ -209,11 +209,14 @@ def lt_hybrid8_step(tensors: TensorList, block: int, hp: HParams, d_sqnorm: Opti
                                 None if d_status is None else d_status.data_ptr(), _stream(stream)))
 
 
-def lt_step_state_advance(d_state: torch.Tensor, hp: HParams, stream=None) -> None:
-    """d_state: 16 bytes of device memory (an lt_step_state), zeroed once by the caller."""
+def lt_step_state_advance(d_state: torch.Tensor, hp: HParams, d_sqnorm: Optional[torch.Tensor] = None, stream=None) -> None:
+    """d_state: 16 bytes of device memory (an lt_step_state), zeroed once by the caller. With d_sqnorm the
+    count stays where it is when the norm is not finite (the step that follows is skipped)."""
     assert d_state.is_cuda and d_state.numel() * d_state.element_size() >= 16
     h = hp.c()
-    _check("lt_step_state_advance", _lib.lt_step_state_advance(d_state.data_ptr(), C.byref(h), _stream(stream)))
+    _check("lt_step_state_advance",
+           _lib.lt_step_state_advance(d_state.data_ptr(), C.byref(h),
+                                      None if d_sqnorm is None else d_sqnorm.data_ptr(), _stream(stream)))
 
 
 def lt_hybrid8_step_graph(tensors: TensorList, block: int, hp: HParams, d_state: torch.Tensor,
@@ -250,7 +253,7 @@ class GraphedHybrid8Optimizer:
         for ch in self.chunks:
             lt_grad_sqnorm_multi(ch, self.sqnorm, self.workspace)
         lt_skip_count_update(self.sqnorm, self.skip_count)
-        lt_step_state_advance(self.state, self.hp)
+        lt_step_state_advance(self.state, self.hp, self.sqnorm)
         for ch in self.chunks:
             lt_hybrid8_step_graph(ch, self.block, self.hp, self.state, self.sqnorm, self.status)
 
@@ -292,3 +295,16 @@ class Hybrid8Optimizer:
         lt_skip_count_update(self.sqnorm, self.skip_count)
         for ch in self.chunks:
             lt_hybrid8_step(ch, self.block, self.hp, self.sqnorm, self.status)
+
+    def settle_skipped_step(self) -> bool:
+        """Reads the status word (a host synchronisation, so the caller picks the moment: typically where it
+        reads the loss). If the last step was skipped for a non-finite norm, the step count goes back by one,
+        so that skipped steps do not count towards the bias corrections, and the skip bit is cleared.
+        Returns whether a step had been skipped. Call it after every step that may have been skipped: the
+        host forms the step scalars from this count, and the bit does not say how many steps set it."""
+        st = int(self.status.item())
+        if st & 1:
+            self.t -= 1
+            self.status.fill_(st & ~1)
+            return True
+        return False

@@ -143,8 +143,9 @@ int launch(const StepParams& p, int sm_count, cudaStream_t s) {
 
 }  // namespace
 
-__global__ void step_state_advance_kernel(lt_step_state* st, float lr, float beta1, float beta2) {
+__global__ void step_state_advance_kernel(lt_step_state* st, float lr, float beta1, float beta2, const double* sqnorm) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (sqnorm != nullptr && !isfinite(*sqnorm)) return;   // the coming step is skipped: it does not count
     const int64_t t = st->step + 1;
     const double bc1 = 1.0 - pow((double)beta1, (double)t);
     const double bc2 = 1.0 - pow((double)beta2, (double)t);
@@ -153,8 +154,9 @@ __global__ void step_state_advance_kernel(lt_step_state* st, float lr, float bet
     st->inv_sqrt_bc2 = (float)(1.0 / sqrt(bc2));
 }
 
-int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, cudaStream_t s) {
-    step_state_advance_kernel<<<1, 32, 0, s>>>(d_state, lr, beta1, beta2);
+int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, const double* d_sqnorm,
+                              cudaStream_t s) {
+    step_state_advance_kernel<<<1, 32, 0, s>>>(d_state, lr, beta1, beta2, d_sqnorm);
     return cudaGetLastError() == cudaSuccess ? LT_OK : LT_ERR_CUDA;
 }
 

@@ -283,7 +283,7 @@ int lt_hybrid8_state_init(const lt_tensor* tensors, int32_t n, int32_t block, lt
 
 int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
                          void* d_workspace, int64_t workspace_bytes, lt_stream stream) {
-    int rc = validate_tensors(tensors, n, NEED_GRAD);
+    int rc = validate_grads(tensors, n, nullptr);
     if (rc != LT_OK) return rc;
     if (!d_sqnorm) return LT_ERR_INVALID_ARG;
     if (!aligned(d_sqnorm, 8)) return LT_ERR_ALIGNMENT;
@@ -297,27 +297,8 @@ int lt_grad_sqnorm_multi(const lt_tensor* tensors, int32_t n, double* d_sqnorm,
     P.out = d_sqnorm;
     int32_t i = 0;
     while (i < n) {
-        int cnt = 0;
-        int64_t items = 0;
-        while (i < n && cnt < kCap) {
-            const lt_tensor& x = tensors[i];
-            if (x.numel == 0) { ++i; continue; }
-            const uintptr_t a = (uintptr_t)x.grad;
-            const int lead = (int)(a & 15);
-            const int64_t span = lead + x.numel * esize(x.grad_dtype);
-            const int64_t it = (span + kNormItemBytes - 1) / kNormItemBytes;
-            if (items + it > 0x7fffffff) break;
-            NormDesc& d = P.t[cnt];
-            d.base16 = (const void*)(a - lead);
-            d.span_bytes = span;
-            items += it;
-            d.item_end = (int32_t)items;
-            d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
-            ++cnt; ++i;
-        }
-        if (cnt == 0) continue;
-        P.n = cnt;
-        P.total_items = (int32_t)items;
+        pack_norm(tensors, n, &i, &P);
+        if (P.n == 0) continue;
         // the arrival counter must start at zero whatever an earlier (possibly failed) launch left
         if (cudaMemsetAsync(P.ticket, 0, 256, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
         if ((rc = launch_sqnorm(P, dev->sm_count, (cudaStream_t)stream)) != LT_OK) return rc;
@@ -334,7 +315,7 @@ static int step_impl(const lt_tensor* tensors, int32_t n, int32_t block, const l
     if (use_state) {
         if (!d_state) return LT_ERR_INVALID_ARG;
         if (!aligned(d_state, 8)) return LT_ERR_ALIGNMENT;
-        hp_local.step = 1;   // the largest step size any count can give (rule below); the kernels read the real scalars
+        hp_local.step = 1;   // any valid count: the kernels read the real scalars from the device
     }
     const lt_hparams* hp = &hp_local;
     int rc = validate_tensors(tensors, n, NEED_GRAD | NEED_PARAM | NEED_STATE);
@@ -400,12 +381,12 @@ int lt_hybrid8_step_graph(const lt_tensor* tensors, int32_t n, int32_t block, co
     return step_impl(tensors, n, block, hp, d_state, true, d_sqnorm, d_status, stream);
 }
 
-int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, lt_stream stream) {
+int lt_step_state_advance(lt_step_state* d_state, const lt_hparams* hp, const double* d_sqnorm, lt_stream stream) {
     if (!d_state || !hp) return LT_ERR_INVALID_ARG;
-    if (!aligned(d_state, 8)) return LT_ERR_ALIGNMENT;
+    if (!aligned(d_state, 8) || (d_sqnorm && !aligned(d_sqnorm, 8))) return LT_ERR_ALIGNMENT;
     if (!(hp->beta1 >= 0.0f && hp->beta1 < 1.0f) || !(hp->beta2 >= 0.0f && hp->beta2 < 1.0f) || !std::isfinite(hp->lr))
         return LT_ERR_INVALID_ARG;
-    return launch_step_state_advance(d_state, hp->lr, hp->beta1, hp->beta2, (cudaStream_t)stream);
+    return launch_step_state_advance(d_state, hp->lr, hp->beta1, hp->beta2, d_sqnorm, (cudaStream_t)stream);
 }
 
 }  // extern "C"

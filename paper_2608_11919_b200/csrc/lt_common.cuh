@@ -94,7 +94,13 @@ int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s);   // tensors with fp32 moments
 constexpr int kAdamw32Item = 2048;   // elements per work item of that kernel (items restart at every tensor)
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
-int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, cudaStream_t s);
+// Host-side checks of the fields the norm kernels read (grad, grad_dtype, numel); *live = non-empty tensors.
+int validate_grads(const lt_tensor* t, int32_t n, int* live);
+// Packs tensors [*i, n) into one launch's descriptors: at most kCap non-empty tensors and fewer than 2^31
+// work items; advances *i past what it took. P->n == 0 when nothing was left. slot = index in the list.
+void pack_norm(const lt_tensor* t, int32_t n, int32_t* i, NormParams* P);
+int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, float beta2, const double* d_sqnorm,
+                              cudaStream_t s);
 int upload_tables(cudaStream_t s);
 
 #ifndef LT_NORM_THREADS

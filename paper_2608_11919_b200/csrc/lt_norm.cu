@@ -134,6 +134,48 @@ __global__ void __launch_bounds__(kNormThreads, kNormCtasPerSm) sqnorm_kernel(co
     }
 }
 
+int validate_grads(const lt_tensor* t, int32_t n, int* live) {
+    if (n < 0 || (n > 0 && t == nullptr)) return LT_ERR_INVALID_ARG;
+    int cnt = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const lt_tensor& x = t[i];
+        if (x.numel < 0) return LT_ERR_INVALID_ARG;
+        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;   // keeps per-launch item counts in int32
+        if (x.numel == 0) continue;
+        if ((x.grad_dtype != LT_F32 && x.grad_dtype != LT_BF16) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
+        if (((uintptr_t)x.grad % (x.grad_dtype == LT_F32 ? 4 : 2)) != 0) return LT_ERR_ALIGNMENT;
+        ++cnt;
+    }
+    if (live) *live = cnt;
+    return LT_OK;
+}
+
+void pack_norm(const lt_tensor* t, int32_t n, int32_t* i, NormParams* P) {
+    int cnt = 0;
+    int64_t items = 0;
+    while (*i < n && cnt < kCap) {
+        const lt_tensor& x = t[*i];
+        if (x.numel == 0) { ++*i; continue; }
+        // the kernel reads whole 16-byte vectors: the span starts at the address rounded down to 16 bytes
+        const uintptr_t a = (uintptr_t)x.grad;
+        const int lead = (int)(a & 15);
+        const int64_t span = lead + x.numel * (x.grad_dtype == LT_F32 ? 4 : 2);
+        const int64_t it = (span + kNormItemBytes - 1) / kNormItemBytes;
+        if (items + it > 0x7fffffff) break;   // next launch; one tensor alone always fits (numel <= 2^38)
+        NormDesc& d = P->t[cnt];
+        d.base16 = (const void*)(a - lead);
+        d.span_bytes = span;
+        items += it;
+        d.item_end = (int32_t)items;
+        d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
+        d.slot = *i;
+        d.pad = 0;
+        ++cnt; ++*i;
+    }
+    P->n = cnt;
+    P->total_items = (int32_t)items;
+}
+
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s) {
     int grid = kNormCtasPerSm * sm_count;
     if (grid > kNormMaxCtas) grid = kNormMaxCtas;
@@ -201,45 +243,18 @@ __global__ void skip_count_kernel(const double* sqnorm, int32_t* count) {
 
 extern "C" int lt_grad_sqnorm_per_tensor(const lt_tensor* tensors, int32_t n, double* d_out, lt_stream stream) {
     using namespace lt;
-    if (n < 0 || (n > 0 && tensors == nullptr) || (n > 0 && d_out == nullptr)) return LT_ERR_INVALID_ARG;
-    if (((uintptr_t)d_out & 7) != 0) return LT_ERR_ALIGNMENT;
-    for (int32_t i = 0; i < n; ++i) {
-        const lt_tensor& x = tensors[i];
-        if (x.numel < 0) return LT_ERR_INVALID_ARG;
-        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;
-        if (x.numel == 0) continue;
-        if ((x.grad_dtype != LT_F32 && x.grad_dtype != LT_BF16) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
-        if (((uintptr_t)x.grad % (x.grad_dtype == LT_F32 ? 4 : 2)) != 0) return LT_ERR_ALIGNMENT;
-    }
-    DeviceInfo* dev = nullptr;
-    int rc = ensure_device((cudaStream_t)stream, &dev);
+    int rc = validate_grads(tensors, n, nullptr);
     if (rc != LT_OK) return rc;
+    if (n > 0 && d_out == nullptr) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_out & 7) != 0) return LT_ERR_ALIGNMENT;
+    DeviceInfo* dev = nullptr;
+    if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
     NormParams P;
     P.ticket = nullptr; P.partials = nullptr; P.out = d_out;
     int32_t i = 0;
     while (i < n) {
-        int cnt = 0;
-        int64_t items = 0;
-        while (i < n && cnt < kCap) {
-            const lt_tensor& x = tensors[i];
-            if (x.numel == 0) { ++i; continue; }
-            const uintptr_t a = (uintptr_t)x.grad;
-            const int lead = (int)(a & 15);
-            const int64_t span = lead + x.numel * (x.grad_dtype == LT_F32 ? 4 : 2);
-            const int64_t it = (span + kNormItemBytes - 1) / kNormItemBytes;
-            if (items + it > 0x7fffffff) break;
-            NormDesc& d = P.t[cnt];
-            d.base16 = (const void*)(a - lead);
-            d.span_bytes = span;
-            items += it;
-            d.item_end = (int32_t)items;
-            d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
-            d.slot = i;
-            ++cnt; ++i;
-        }
-        if (cnt == 0) continue;
-        P.n = cnt;
-        P.total_items = (int32_t)items;
+        pack_norm(tensors, n, &i, &P);
+        if (P.n == 0) continue;
         int grid = kNormCtasPerSm * dev->sm_count;
         if (grid > P.total_items) grid = P.total_items;
         sqnorm_per_tensor_kernel<<<grid, kNormThreads, 0, (cudaStream_t)stream>>>(P);
@@ -290,49 +305,26 @@ int noalloc_scratch(void** out) {
 
 extern "C" int lt_grad_sqnorm_multi_noalloc(const lt_tensor* tensors, int32_t n, double* d_sqnorm, lt_stream stream) {
     using namespace lt;
-    if (n < 0 || (n > 0 && tensors == nullptr) || d_sqnorm == nullptr) return LT_ERR_INVALID_ARG;
-    if (((uintptr_t)d_sqnorm & 7) != 0) return LT_ERR_ALIGNMENT;
     int live = 0;
-    for (int32_t i = 0; i < n; ++i) {
-        const lt_tensor& x = tensors[i];
-        if (x.numel < 0) return LT_ERR_INVALID_ARG;
-        if (x.numel > ((int64_t)1 << 38)) return LT_ERR_UNSUPPORTED;
-        if (x.numel == 0) continue;
-        if ((x.grad_dtype != LT_F32 && x.grad_dtype != LT_BF16) || x.grad == nullptr) return LT_ERR_INVALID_ARG;
-        if (((uintptr_t)x.grad % (x.grad_dtype == LT_F32 ? 4 : 2)) != 0) return LT_ERR_ALIGNMENT;
-        ++live;
-    }
+    int rc = validate_grads(tensors, n, &live);
+    if (rc != LT_OK) return rc;
+    if (d_sqnorm == nullptr) return LT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_sqnorm & 7) != 0) return LT_ERR_ALIGNMENT;
     if (live > LT_NOALLOC_MAX_TENSORS) return LT_ERR_WORKSPACE;   // beyond what one launch over the fixed scratch covers
     if (live == 0) return LT_OK;
+    NormParams P;
+    int32_t i = 0;
+    pack_norm(tensors, n, &i, &P);
+    while (i < n && tensors[i].numel == 0) ++i;
+    if (i < n) return LT_ERR_UNSUPPORTED;     // 2^31 work items or more: not one launch (nothing has been touched yet)
 
     DeviceInfo* dev = nullptr;
-    int rc = ensure_device((cudaStream_t)stream, &dev);
-    if (rc != LT_OK) return rc;
+    if ((rc = ensure_device((cudaStream_t)stream, &dev)) != LT_OK) return rc;
     void* scratch = nullptr;
     if ((rc = noalloc_scratch(&scratch)) != LT_OK) return rc;
-
-    NormParams P;
     P.ticket = (unsigned int*)scratch;
     P.partials = (double*)((char*)scratch + 256);
     P.out = d_sqnorm;
-    int cnt = 0;
-    int64_t items = 0;
-    for (int32_t i = 0; i < n; ++i) {
-        const lt_tensor& x = tensors[i];
-        if (x.numel == 0) continue;
-        const uintptr_t a = (uintptr_t)x.grad;
-        const int lead = (int)(a & 15);
-        const int64_t span = lead + x.numel * (x.grad_dtype == LT_F32 ? 4 : 2);
-        items += (span + kNormItemBytes - 1) / kNormItemBytes;
-        if (items > 0x7fffffff) return LT_ERR_UNSUPPORTED;
-        NormDesc& d = P.t[cnt++];
-        d.base16 = (const void*)(a - lead);
-        d.span_bytes = span;
-        d.item_end = (int32_t)items;
-        d.lead_f32 = lead | ((x.grad_dtype == LT_F32 ? 1 : 0) << 8);
-    }
-    P.n = cnt;
-    P.total_items = (int32_t)items;
     // the array keeps what the last call left: the arrival counter must start at zero
     if (cudaMemsetAsync(P.ticket, 0, 256, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return LT_ERR_CUDA; }
     int grid = kNormCtasPerSm * dev->sm_count;

@@ -1,5 +1,5 @@
 """Host-resident variant: parameters, gradients and optimizer state live in pinned HOST memory (the
-paper's layout, Sec. 3.5: "keeps parameters and optimizer states in CPU memory") and are streamed through
+paper's layout, Sec. 3.5: master parameters and optimizer states stay in CPU memory) and are streamed through
 the same kernels chunk by chunk, with copies and compute overlapped on three streams.
 
 Per optimizer step:
@@ -7,8 +7,13 @@ Per optimizer step:
           the device if `keep_grads` so that pass 2 does not send them again)
   pass 2  every chunk: parameters + state H2D -> lt_hybrid8_step -> parameters + state D2H
           (two staging slots: chunk k+1 is copied in while chunk k is updated and chunk k-1 is copied out)
-The bound is the host link, not HBM. This module is plumbing only: every arithmetic step is in the
-library's kernels.
+The bound is the host link, not HBM: per parameter 8 bytes go in (gradient, fp32 parameter, two codes) and 6
+come back, and while both directions are busy each gets less than it gets alone, so the floor of a step is
+(bytes out) / (per-direction rate with both busy) + (bytes in - bytes out) / (one-direction rate). This module
+is plumbing only: every arithmetic step is in the library's kernels.
+
+The host side is a `HostTensors`: per-tensor pinned tensors the caller owns (a trainer's own master weights,
+gradients and state), or the flat buffers of a synthetic workload through `HostTensors.from_buffers`.
 """
 from __future__ import annotations
 
@@ -17,16 +22,55 @@ from typing import List, Optional, Sequence
 import torch
 
 from . import binding as B
-from . import workloads as W
 
 _KEYS = ("param", "m_code", "v_code", "m_absmax", "v_absmax")
+
+
+class HostTensors:
+    """The host side of the optimizer: one pinned CPU tensor per model tensor and kind.
+
+    params[t], grads[t]: [numel_t]; m_state[t], v_state[t]: uint8 [numel_t] codes, or float32 [numel_t] moments for
+    a tensor with plain fp32 state; m_absmax[t], v_absmax[t]: float32 [ceil(numel_t / block)] (ignored, may be
+    None, for fp32-state tensors). All parameters share one dtype, all gradients share one dtype. Tensors that
+    lie back to back in host memory are copied with one transfer."""
+
+    def __init__(self, params, grads, m_state, v_state, m_absmax, v_absmax):
+        n = len(params)
+        assert all(len(x) == n for x in (grads, m_state, v_state, m_absmax, v_absmax))
+        self._t = {"param": list(params), "grad": list(grads), "m_code": list(m_state), "v_code": list(v_state),
+                   "m_absmax": list(m_absmax), "v_absmax": list(v_absmax)}
+        self.sizes = [int(p.numel()) for p in params]
+        self.f32 = [m.dtype == torch.float32 for m in m_state]
+        self.param_dtype = params[0].dtype if n else torch.float32
+        self.grad_dtype = grads[0].dtype if n else torch.bfloat16
+        for t in range(n):
+            assert params[t].dtype == self.param_dtype and grads[t].dtype == self.grad_dtype
+            assert grads[t].numel() == self.sizes[t] and m_state[t].numel() == self.sizes[t]
+            for k in ("param", "grad", "m_code", "v_code"):
+                x = self._t[k][t]
+                assert x.device.type == "cpu" and x.is_contiguous() and (x.numel() == 0 or x.is_pinned()), \
+                    "host tensors must be contiguous pinned CPU memory"
+        self._empty = torch.empty(0, dtype=torch.float32)
+
+    @classmethod
+    def from_buffers(cls, buf) -> "HostTensors":
+        """Views of the flat host buffers of a `workloads.Buffers` (allocated with pin=True)."""
+        n = len(buf.spec.sizes)
+        return cls(*[[buf.view(k, t) for t in range(n)]
+                     for k in ("param", "grad", "m_code", "v_code", "m_absmax", "v_absmax")])
+
+    def view(self, key: str, t: int) -> torch.Tensor:
+        x = self._t[key][t]
+        if key in ("m_absmax", "v_absmax") and (self.f32[t] or x is None):
+            return self._empty
+        return x
 
 
 class _Slot:
     """Device staging for one chunk: flat buffers big enough for the largest chunk."""
 
-    def __init__(self, host: W.Buffers, max_elems: int, max_blocks: int, max_f32: int, device):
-        spec = host.spec
+    def __init__(self, host: HostTensors, max_elems: int, max_blocks: int, max_f32: int, device):
+        spec = host
         kw = dict(device=device)
         self.param = torch.empty(max(max_elems, 1), dtype=spec.param_dtype, **kw)
         self.grad = torch.empty(max(max_elems, 1), dtype=spec.grad_dtype, **kw)
@@ -43,13 +87,17 @@ class _Slot:
 
 
 class HostResidentOptimizer:
-    def __init__(self, host: W.Buffers, block: int, hp: B.HParams, chunks: Sequence[Sequence[int]],
-                 device="cuda:0", keep_grads: bool = True):
-        assert host.device.type == "cpu" and host.param.is_pinned(), "host buffers must be pinned CPU memory"
+    def __init__(self, host, block: int, hp: B.HParams, chunks: Sequence[Sequence[int]],
+                 device="cuda:0", keep_grads: bool = True, n_slots: int = 3):
+        """host: a HostTensors (or a pinned `workloads.Buffers`, wrapped here). chunks: lists of tensor indices,
+        updated one chunk at a time under one global clip norm. n_slots device staging buffers (of the largest
+        chunk's size) let copy-in, update and copy-out of neighbouring chunks overlap."""
+        if not isinstance(host, HostTensors):
+            host = HostTensors.from_buffers(host)
         self.host, self.block, self.hp = host, int(block), hp
         self.device = torch.device(device)
         self.chunks = [list(c) for c in chunks if len(c)]
-        spec, a = host.spec, host.spec.align_elems
+        spec, a = host, 16          # tensors start on 16-element boundaries inside the staging buffers
         # placement of every tensor inside its chunk's staging buffers
         self.place = {}
         max_e = max_b = max_f = 0
@@ -66,9 +114,15 @@ class HostResidentOptimizer:
                 else:
                     e8 += s; b += nb
             max_e, max_b, max_f = max(max_e, e), max(max_b, b), max(max_f, f)
-        self.slots = [_Slot(host, max_e, max_b, max_f, self.device) for _ in range(2)]
+        self.slots = [_Slot(host, max_e, max_b, max_f, self.device) for _ in range(max(2, int(n_slots)))]
+        self.n_slots = len(self.slots)
         self.keep_grads = keep_grads
-        self.dev_grad = torch.empty(host.grad.numel(), dtype=spec.grad_dtype, device=self.device) if keep_grads else None
+        self.goff, o = [], 0       # placement of every tensor's gradient in the device-resident gradient buffer
+        for sz in spec.sizes:
+            o = (o + a - 1) // a * a
+            self.goff.append(o)
+            o += sz
+        self.dev_grad = torch.empty(max(o, 1), dtype=spec.grad_dtype, device=self.device) if keep_grads else None
         self.sqnorm = torch.zeros(1, dtype=torch.float64, device=self.device)
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.workspace = torch.empty(B.lt_workspace_bytes(), dtype=torch.uint8, device=self.device)
@@ -111,10 +165,10 @@ class HostResidentOptimizer:
     # device view of tensor t inside a slot
     def _dev(self, sl: _Slot, key: str, t: int) -> torch.Tensor:
         e, e8, b, f = self.place[t]
-        s = self.host.spec.sizes[t]
+        s = self.host.sizes[t]
         f32 = self.host.f32[t]
         if key == "grad" and self.keep_grads:
-            return self.dev_grad[self.host.off[t]: self.host.off[t] + s]
+            return self.dev_grad[self.goff[t]: self.goff[t] + s]
         if key in ("param", "grad"):
             return getattr(sl, key)[e: e + s]
         if key in ("m_code", "v_code"):
@@ -148,18 +202,19 @@ class HostResidentOptimizer:
         # pass 1: gradients in, norm
         self.h2d.wait_stream(main)
         for ci, c in enumerate(self.chunks):
-            sl = self.slots[ci % 2]
+            sl = self.slots[ci % self.n_slots]
             with torch.cuda.stream(self.h2d):
-                self.h2d.wait_event(sl.stepped if not self.keep_grads else sl.drained)
-                for d, h in self.plan[(ci, ci % 2, "grad")]:
+                if not self.keep_grads:
+                    self.h2d.wait_event(sl.stepped)     # the slot's previous gradients have been read
+                for d, h in self.plan[(ci, ci % self.n_slots, "grad")]:
                     h2d += self._copy(d, h)
                 sl.filled.record(self.h2d)
             main.wait_event(sl.filled)
-            B.lt_grad_sqnorm_multi(self.lists[(ci, ci % 2)], self.sqnorm, self.workspace)
+            B.lt_grad_sqnorm_multi(self.lists[(ci, ci % self.n_slots)], self.sqnorm, self.workspace)
             sl.stepped.record(main)
         # pass 2: parameters and state in, step, out
         for ci, c in enumerate(self.chunks):
-            si = ci % 2
+            si = ci % self.n_slots
             sl = self.slots[si]
             with torch.cuda.stream(self.h2d):
                 self.h2d.wait_event(sl.drained)         # the slot's previous results have left

@@ -173,8 +173,11 @@ class Buffers:
     param / grad. Tensors with 8-bit state own [off8[t], ...) of m_code / v_code and [boff[t], boff[t]+nb[t])
     of the two scale arrays; tensors with fp32 state own [off32[t], ...) of m_f32 / v_f32."""
 
-    def __init__(self, spec: Spec, block: int, device, pin: bool = False):
+    def __init__(self, spec: Spec, block: int, device, pin: bool = False, guard_bytes: int = 0):
+        """guard_bytes > 0: every flat buffer is followed by that many bytes of a fixed pattern which
+        check_guards() verifies (a write past the end of the last tensor shows up there)."""
         self.spec, self.block, self.device = spec, int(block), torch.device(device)
+        self._guards = []
         a = spec.align_elems
         self.f32 = list(spec.state_f32) if spec.state_f32 is not None else [False] * len(spec.sizes)
         self.off, self.boff, self.off8, self.off32 = [], [], [], []
@@ -193,14 +196,28 @@ class Buffers:
         kw = dict(device=self.device)
         if pin and self.device.type == "cpu":
             kw["pin_memory"] = True
-        self.param = torch.empty(max(o, 1), dtype=spec.param_dtype, **kw)
-        self.grad = torch.empty(max(o, 1), dtype=spec.grad_dtype, **kw)
-        self.m_code = torch.empty(max(o8, 1), dtype=torch.uint8, **kw)
-        self.v_code = torch.empty(max(o8, 1), dtype=torch.uint8, **kw)
-        self.m_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
-        self.v_absmax = torch.empty(max(b, 1), dtype=torch.float32, **kw)
-        self.m_f32 = torch.empty(max(o32, 1), dtype=torch.float32, **kw)
-        self.v_f32 = torch.empty(max(o32, 1), dtype=torch.float32, **kw)
+        def flat(n, dtype):
+            n = max(n, 1)
+            if guard_bytes <= 0:
+                return torch.empty(n, dtype=dtype, **kw)
+            es = torch.empty(0, dtype=dtype).element_size()
+            raw = torch.empty(n * es + guard_bytes, dtype=torch.uint8, **kw)
+            raw[n * es:] = 0xA5
+            self._guards.append(raw[n * es:])
+            return raw[:n * es].view(dtype)
+
+        self.param = flat(o, spec.param_dtype)
+        self.grad = flat(o, spec.grad_dtype)
+        self.m_code = flat(o8, torch.uint8)
+        self.v_code = flat(o8, torch.uint8)
+        self.m_absmax = flat(b, torch.float32)
+        self.v_absmax = flat(b, torch.float32)
+        self.m_f32 = flat(o32, torch.float32)
+        self.v_f32 = flat(o32, torch.float32)
+
+    def check_guards(self) -> None:
+        for i, g in enumerate(self._guards):
+            assert bool((g == 0xA5).all()), f"guard bytes after flat buffer {i} were overwritten"
 
     def view(self, which: str, t: int) -> torch.Tensor:
         size = self.spec.sizes[t]

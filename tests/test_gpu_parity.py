@@ -29,7 +29,7 @@ def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True,
     resync: after every comparison the oracle takes over the GPU's parameters, so that each step is
     compared from identical inputs (the state is compared for identity anyway)."""
     torch.cuda.set_device(0)
-    buf = W.Buffers(spec, block, DEV)
+    buf = W.Buffers(spec, block, DEV, guard_bytes=256)
     W.fill_params(buf)
     tl = L.TensorList.from_buffers(buf)
     hp = L.HParams(max_norm=spec.max_norm, **(hp_kw or {}))
@@ -61,6 +61,7 @@ def run_free(spec, block, steps, hp_kw=None, chunks=None, check_every_step=True,
         ohp.step = k
         assert parallel_oracle_step(ots, block, ohp, S) == 0
         assert int(opt.status.item()) == 0
+        buf.check_guards()                       # nothing was written past the end of any flat buffer
         if check_every_step or k == steps:
             st = compare(buf, ots, slices)
             st.norm_rel = abs(S_gpu - S) / S if S else 0.0
@@ -241,6 +242,45 @@ def test_nonfinite_gradient_skips_step(bad):
     torch.cuda.synchronize()
     assert int(opt.status.item()) == 0
     assert not torch.equal(buf.param, before["param"])
+
+
+@pytest.mark.parametrize("graphed", [False, True])
+def test_a_skipped_step_does_not_count_towards_the_bias_corrections(graphed):
+    """Steps 1, 2(non-finite: skipped), 3 must leave exactly what steps 1, 2 of a run without the bad step leave:
+    the step count that forms lr / (1 - beta1^t) and 1 / sqrt(1 - beta2^t) does not advance on a skipped step
+    (device-side in the graphed driver; settle_skipped_step() in the eager one)."""
+    torch.cuda.set_device(0)
+    spec = W.ragged_spec(n_tensors=30, max_numel=1 << 14, seed=12)
+    cls = L.GraphedHybrid8Optimizer if graphed else L.Hybrid8Optimizer
+    bufs = []
+    for with_bad_step in (False, True):
+        buf = W.Buffers(spec, 2048, DEV)
+        W.fill_params(buf)
+        opt = cls(L.TensorList.from_buffers(buf), 2048, L.HParams(max_norm=0.5, lr=1e-3))
+        opt.init_state()
+        W.fill_grads(buf, 1)
+        opt.step()
+        if with_bad_step:
+            W.fill_grads(buf, 7)
+            buf.view("grad", 5)[0] = float("nan")
+            opt.step()
+            torch.cuda.synchronize()
+            assert int(opt.status.item()) & 1
+            if graphed:
+                assert int(opt.state.cpu()[0]) == 1 and int(opt.skip_count.item()) == 1
+                opt.status.zero_()
+            else:
+                assert opt.settle_skipped_step() and opt.t == 1 and not opt.settle_skipped_step()
+        W.fill_grads(buf, 2)
+        opt.step()
+        torch.cuda.synchronize()
+        assert int(opt.status.item()) == 0
+        bufs.append(buf)
+    for key in ("param", "m_code", "v_code", "m_absmax", "v_absmax"):
+        a, b = getattr(bufs[0], key), getattr(bufs[1], key)
+        if a.dtype == torch.float32:
+            a, b = a.view(torch.int32), b.view(torch.int32)
+        assert torch.equal(a, b), key
 
 
 def test_byte_zero_state_equals_value_zero_state():

@@ -540,3 +540,24 @@ def test_fp32_state_tensors_in_the_step_equal_the_pinned_fp32_mode():
     z = O.OracleTensor(p0.copy(), np.zeros(n, np.uint16), 4096, m_code=np.ones(n, np.float32), v_code=np.ones(n, np.float32))
     O.state_init([z], 4096)
     assert not z.m_code.any() and not z.v_code.any()
+
+
+def test_oracle_is_clean_under_address_and_ub_sanitizers(tmp_path):
+    """The oracle compiled with AddressSanitizer and UndefinedBehaviorSanitizer runs its whole path (state init,
+    norm, steps with both quantizers, skip) over exactly-sized heap arrays of awkward lengths without a report."""
+    import shutil
+    import subprocess
+    if shutil.which("g++") is None:
+        pytest.skip("no g++")
+    here = os.path.dirname(os.path.abspath(__file__))
+    exe = str(tmp_path / "oracle_sanitized")
+    cmd = ["g++", "-O1", "-g", "-std=c++17", "-ffp-contract=off", "-fsanitize=address,undefined",
+           "-fno-sanitize-recover=all", "-o", exe, os.path.join(here, "oracle_sanitizer_driver.cpp")]
+    built = subprocess.run(cmd, capture_output=True, text=True)
+    if built.returncode != 0 and "sanitize" in (built.stderr or "") and "cannot find" in built.stderr:
+        pytest.skip("sanitizer runtime not installed")
+    assert built.returncode == 0, built.stderr[-2000:]
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300,
+                         env=dict(os.environ, ASAN_OPTIONS="detect_leaks=1", UBSAN_OPTIONS="print_stacktrace=1"))
+    assert run.returncode == 0, (run.stdout + run.stderr)[-3000:]
+    assert "sanitizer run clean" in run.stdout
