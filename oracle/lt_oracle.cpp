@@ -5,10 +5,11 @@
 // table or constant generator with the CUDA library; the CUDA library never calls it.
 //
 // What it follows. The paper (Sec. 3.5, "Hybrid 8-bit operator") describes the operator in words:
-// a slice of the Adam moments is held as 8-bit codes with block-wise scales, the update
-// dequantizes, applies an AdamW update, and requantizes; a fast clip computes per-tensor norms,
-// aggregates one global norm and applies one scale; non-finite gradients are skipped (training
-// configuration table, "Safety checks" row); hyper-parameters come from the same table
+// a slice of the Adam moments is held as 8-bit codes with one scale per block, the update
+// decodes them, takes an AdamW step and encodes them again; the clip takes a norm per tensor,
+// combines these into one global norm and multiplies every gradient by one factor; a step whose
+// gradients are not finite is left out (training-configuration table, safety-checks row);
+// hyper-parameters come from the same table
 // (beta1 0.9, beta2 0.999, eps 1e-8, lr 1e-5, weight decay 0.01, max grad norm 1.0); block size
 // 4096 comes from the variant-configuration table. The paper prints no formulas for the
 // quantization map, tie handling, epsilon placement or rounding, so this file takes one written
