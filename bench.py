@@ -110,20 +110,9 @@ def build_workload(name: str, block: int, device, shard=None):
     import torch
     import paper_2608_11919_b200 as L
     from paper_2608_11919_b200 import workloads as W
-    from paper_2608_11919_b200.sharding import partition_blocks
     spec = W.SPECS[name]()
-    pieces = None
     if shard is not None:
-        rank, world = shard
-        mine = partition_blocks(spec.sizes, block, world)[rank]
-        # the rank allocates only the tensors it touches; a tensor cut by the partition keeps its owned blocks
-        idx = sorted({t for t, _, _ in mine})
-        pos = {t: i for i, t in enumerate(idx)}
-        full = spec
-        spec = W.subset_spec(full, idx, suffix=f"[rank {rank}/{world}]")
-        spec.sizes = [0] * len(idx)
-        for t, b0, nb in mine:      # pieces of one tensor are consecutive, so the owned part is one run
-            spec.sizes[pos[t]] += min(full.sizes[t], (b0 + nb) * block) - b0 * block
+        spec = W.shard_spec(spec, block, shard[0], shard[1])
     buf = W.Buffers(spec, block, device)
     W.fill_params(buf)
     W.fill_grads(buf, 1)
@@ -476,6 +465,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-alt-block", action="store_true", help="skip the second run at the other block size")
+    ap.add_argument("--force-dist", action="store_true",
+                    help="initialise the process group even with one rank (runs the N > 1 code path on one GPU)")
     ap.add_argument("--host-resident", default="3b,7b",
                     help="workloads of the host-resident end-to-end run (comma separated), or 'none'")
     ap.add_argument("--cpu-sample", type=int, default=128 << 20, help="params in the oracle's timed sample")
@@ -517,7 +508,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the product path)")
     torch.cuda.set_device(local)
-    dist_on = world > 1
+    dist_on = world > 1 or args.force_dist
     if dist_on:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
     peak, peak_kind = measured_peak_gbs()

@@ -159,6 +159,21 @@ def subset_spec(spec: Spec, indices: Sequence[int], suffix: str = "") -> Spec:
         state_f32=None if spec.state_f32 is None else [spec.state_f32[i] for i in idx])
 
 
+def shard_spec(spec: Spec, block: int, rank: int, world: int) -> Spec:
+    """Rank `rank`'s share of ONE list cut into `world` block-balanced shards (sharding.partition_blocks): the
+    tensors the rank touches, each with the size of the block run the rank owns of it (a rank allocates only
+    what it owns; a tensor cut by the partition appears on both neighbours with its part)."""
+    from .sharding import partition_blocks
+    mine = partition_blocks(spec.sizes, block, world)[rank]
+    idx = sorted({t for t, _, _ in mine})
+    pos = {t: i for i, t in enumerate(idx)}
+    out = subset_spec(spec, idx, suffix=f"[rank {rank}/{world}]")
+    out.sizes = [0] * len(idx)
+    for t, b0, nb in mine:      # the pieces of one tensor are consecutive: the owned part is one run
+        out.sizes[pos[t]] += min(spec.sizes[t], (b0 + nb) * block) - b0 * block
+    return out
+
+
 def layer_groups(spec: Spec, layers_per_group: int = 8) -> List[List[int]]:
     """Tensor indices grouped for chunked update: non-layer tensors first, then runs of layers."""
     groups = [[i for i, l in enumerate(spec.layer_of) if l < 0]]

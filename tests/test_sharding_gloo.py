@@ -44,6 +44,22 @@ def test_block_partition_is_balanced_to_one_block():
             assert max(loads) - min(loads) <= 1
 
 
+def test_shard_specs_cover_one_list():
+    """What `bench.py --scaling strong` gives each rank: together the ranks own every element exactly once."""
+    for spec in (W.qwen3b_spec(), W.dense27b_spec()):
+        for world in (2, 8):
+            shards = [W.shard_spec(spec, BLOCK, r, world) for r in range(world)]
+            assert sum(s.numel for s in shards) == spec.numel
+            loads = [s.n_blocks(BLOCK) for s in shards]
+            assert max(loads) - min(loads) <= 1 and sum(loads) == spec.n_blocks(BLOCK)
+            per_name = {}
+            for s in shards:
+                for n, z in zip(s.names, s.sizes):
+                    per_name[n] = per_name.get(n, 0) + z
+            assert per_name == dict(zip(spec.names, spec.sizes))
+            assert all(len(W.layer_groups(s, 8)) >= 1 for s in shards)
+
+
 def _make(spec, step):
     buf = W.Buffers(spec, BLOCK, "cpu")
     W.fill_params(buf)
