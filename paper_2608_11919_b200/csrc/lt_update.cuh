@@ -64,7 +64,8 @@ __device__ __forceinline__ float param_exact(const StepRegs& r, float p, float m
 //     |p'_approx - p'_defined|  <=  5.5 * 2^-23 |u| + 2^-23 |p'|  =  6.6e-7 |u| + 1.2e-7 |p'|.
 // fp32 parameters: that is below 1e-5 * max(|p'|, |u|) for every input, which is the tolerance fp32
 // parameters are held to (relative to the larger of the result and the update that formed it).
-// bf16 parameters: the rounded results stay within one bf16 ulp (>= 2^-9 |p'|) as long as
+// bf16 parameters: a bf16 ulp is at least 2^-8 |p'|; two values less than half of that apart round to
+// bf16 numbers at most one ulp apart, so the rounded results agree within one ulp as long as
 // 6.6e-7 |u| < 2^-9 |p'|, i.e. |u| < 2950 |p'|. cancel_risk(pn, pd) < 0 flags |p'| < 2^-11 |p * decay|;
 // an element that is not flagged has |u| <= |p * decay| + |p'| <= 2049 |p'|, inside that bound. Flagged
 // elements (about 2 in 10^7) take param_exact.
