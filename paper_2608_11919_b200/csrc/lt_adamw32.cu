@@ -2,10 +2,12 @@
 // the paper's hybrid split, Sec. 3.5): read p, g, m, v, write p, m, v -- 26 bytes per parameter with
 // fp32 parameters and bf16 gradients, a pure HBM stream with no tables and no block exchange.
 //
-// Work item = 2048 consecutive elements of one tensor (items restart at every tensor); 256-thread CTAs
-// walk the items in a grid-stride loop, thread `tid` owning the 4-element groups (k * 256 + tid), k < 2,
-// so every warp-wide access is one contiguous run and all eight 16-byte loads of a thread are in flight
-// together. Moments are formed exactly as written (IEEE fp32, one rounding per operation, no fused
+// Work item = 8192 consecutive elements of one tensor (items restart at every tensor); 256-thread CTAs
+// walk the items in a grid-stride loop, thread `tid` owning the 4-element groups (k * 256 + tid), k < 8,
+// so every warp-wide access is one contiguous run and all 32 loads of a thread (24 of them 16 bytes) are in flight
+// together: measured 6 % faster than two groups per thread, the kernel being bound by memory latency times
+// bytes in flight (four groups +1 %, sixteen -3 % against eight).
+// Moments are formed exactly as written (IEEE fp32, one rounding per operation, no fused
 // multiply-add), so the state matches a plain evaluation bit for bit; the parameter update uses the
 // approximate sqrt/reciprocal unless eps is tiny, as in the 8-bit kernel.
 #include <cuda_bf16.h>
@@ -19,7 +21,13 @@ namespace lt {
 
 namespace {
 
-constexpr int kNT = 256;
+#ifndef LT_A32_NT
+#define LT_A32_NT 256
+#endif
+#ifndef LT_A32_MINB
+#define LT_A32_MINB 1
+#endif
+constexpr int kNT = LT_A32_NT;
 constexpr int kK = kAdamw32Item / (4 * kNT);
 
 // Two elements: moments in place, new parameters returned. GUARD (bf16 parameters on the approximate path):
@@ -45,7 +53,7 @@ __device__ __forceinline__ float update(const StepRegs& r, float p, float g, flo
 }
 
 template <bool PRECISE, bool P_BF16>
-__global__ void __launch_bounds__(kNT) adamw32_kernel(const __grid_constant__ StepParams P) {
+__global__ void __launch_bounds__(kNT, LT_A32_MINB) adamw32_kernel(const __grid_constant__ StepParams P) {
     const int tid = threadIdx.x;
     StepRegs r;
     if (!load_step_regs(P, r)) return;

@@ -92,7 +92,10 @@ const uint32_t* host_lut(bool is_signed, bool full);   // nullptr if the maps do
 int launch_state_init(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_step(const StepParams& p, int block, int sm_count, cudaStream_t s);
 int launch_adamw32(const StepParams& p, int sm_count, cudaStream_t s);   // tensors with fp32 moments
-constexpr int kAdamw32Item = 2048;   // elements per work item of that kernel (items restart at every tensor)
+#ifndef LT_A32_ITEM
+#define LT_A32_ITEM 8192
+#endif
+constexpr int kAdamw32Item = LT_A32_ITEM;   // elements per work item of that kernel (items restart at every tensor)
 int launch_sqnorm(const NormParams& p, int sm_count, cudaStream_t s);
 // Host-side checks of the fields the norm kernels read (grad, grad_dtype, numel); *live = non-empty tensors.
 int validate_grads(const lt_tensor* t, int32_t n, int* live);
@@ -103,10 +106,13 @@ int launch_step_state_advance(lt_step_state* d_state, float lr, float beta1, flo
                               cudaStream_t s);
 int upload_tables(cudaStream_t s);
 
+// Launch shape of the norm kernels: one 1024-thread CTA per SM, eight 16-byte loads per thread and item
+// (128 KiB in flight per SM). Measured on 15 GB of bf16 gradients, sustained: 6.8 TB/s, against 6.2 TB/s for two
+// 512-thread CTAs with four loads per thread (half the bytes in flight), 6.6 for 512 x 8 x 2, 6.9 for 1024 x 10 x 1.
 #ifndef LT_NORM_THREADS
-#define LT_NORM_THREADS 512
-#define LT_NORM_VPT 4
-#define LT_NORM_CTAS 2
+#define LT_NORM_THREADS 1024
+#define LT_NORM_VPT 8
+#define LT_NORM_CTAS 1
 #endif
 constexpr int kNormThreads = LT_NORM_THREADS;
 constexpr int kNormVecPerThread = LT_NORM_VPT;
